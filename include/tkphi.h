@@ -1,0 +1,177 @@
+/*
+ * tkphi.h -- C ABI of libtkphi: decode-step Top-K+phi residual-mass attention
+ * and its prefill summary build, as hand-written CUDA kernels for sm_100a.
+ *
+ * Method (arXiv 2604.05438, "Residual-Mass Accounting for Partial-KV Decoding"):
+ * for one attention layer and each decode query head the library
+ *   (1) scores the query against every mid-region key, s_i = q.k_i / sqrt(d_h)
+ *       (Sec. 3, Eq. full_attention), and selects the K highest-scoring
+ *       mid-region indices K(q) (exhaustive Top-K control selector, Sec. 5.1);
+ *   (2) forms the exact unnormalised terms nu_E, Z_E over E = A U K(q), A the
+ *       sink/tail anchors (Sec. 3, Eq. partition and Eq. exact_terms);
+ *   (3) removes the retrieved tokens' feature contributions from the prefill
+ *       summaries (S, u) (Sec. 4.2, Eq. subtraction);
+ *   (4) evaluates the residual estimate nu_hat_R = S_R phi_q(q),
+ *       Z_hat_R = phi_q(q)^T u_R (Sec. 4.3);
+ *   (5) returns y = (nu_E + nu_hat_R) / (Z_E + Z_hat_R) (Sec. 4.3, Eq. hybrid_merge).
+ * The prefill pass builds S = sum_{i in M} v_i phi_k(k_i)^T, u = sum_{i in M} phi_k(k_i)
+ * over the mid-region M (Sec. 4.1, Eq. natural_cache).
+ *
+ * Feature maps: phi(x) = exp(W x + b - gamma ||x||^2) elementwise, W in R^{r x d};
+ * one map per query head (phi_q) and one per KV head (phi_k) (Sec. 4.1; positivity
+ * by exponentiation, App. C.1).
+ *
+ * General rules
+ *  - Every tensor pointer is a DEVICE pointer unless its comment says "host".
+ *    The caller owns all memory; the library allocates nothing, keeps nothing
+ *    between calls, and enqueues its work on the caller's stream (a
+ *    cudaStream_t passed as void*; NULL is the default stream).
+ *  - Functions return after enqueuing.  The return value reports host-side
+ *    validation and launch errors only; invalid arguments are rejected before
+ *    anything is launched.  tkphi_last_error() gives a message for the last
+ *    failing call of the calling thread.
+ *  - Small per-sequence arrays (cu_seqlens, topk) are passed twice: a host copy
+ *    (validated, used for sizing) and a device copy with the same contents (read
+ *    by the kernels), so that no call needs a device-to-host synchronisation.
+ *  - Inputs must be finite.  Results for NaN/Inf inputs are unspecified.
+ *  - One call processes one attention layer; a model stack is a host loop.
+ */
+#ifndef TKPHI_H
+#define TKPHI_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TKPHI_OK = 0,
+  TKPHI_ERR_INVALID_ARG = -1,  /* bad pointer, size, stride or range */
+  TKPHI_ERR_UNSUPPORTED = -2,  /* legal problem this build has no kernel for */
+  TKPHI_ERR_WORKSPACE = -3,    /* workspace NULL, misaligned or too small */
+  TKPHI_ERR_CUDA = -4,         /* a CUDA runtime/driver call failed */
+  TKPHI_ERR_TIMEOUT = -5       /* a bounded device-side wait ran out (see tkphi_device_status) */
+} tkphi_status;
+
+/* Which entry point a workspace is sized for. */
+enum { TKPHI_WS_BUILD = 0, TKPHI_WS_TOPK_DECODE = 1, TKPHI_WS_DECODE_STEP = 2 };
+
+/* Flags of tkphi_decode_step. */
+enum {
+  TKPHI_FLAG_NONE = 0,
+  TKPHI_FLAG_NOSUB = 1 /* skip the retrieved-token subtraction (the paper's NoSub ablation, Sec. 5.1) */
+};
+
+/*
+ * One attention layer's K/V cache for `batch` ragged sequences (Sec. 3: keys and
+ * values (k_i, v_i), i < L, per KV head).  Sequence b owns cache rows
+ * cu_seqlens[b] .. cu_seqlens[b+1]-1; its prefill length is L_b = cu_seqlens[b+1]
+ * - cu_seqlens[b] >= 1.  Element (head h, row t, dim c) of k is at
+ * k + h*kv_stride_head + t*kv_stride_token + c (in bf16 elements); v uses the
+ * same strides.  Requirements: head_dim in {64, 128}; n_q_heads a multiple of
+ * n_kv_heads with group size <= 8; n_feat in {64, 128}; k and v 16-byte aligned;
+ * both strides multiples of 8 elements; kv_stride_token >= head_dim; total rows
+ * < 2^31.  Query head h_q uses KV head h_q / (n_q_heads / n_kv_heads).
+ * Anchors (Eq. partition): the first n_sink and the last n_tail rows of each
+ * sequence (their union when L_b < n_sink + n_tail); the mid-region is what lies
+ * between, |M_b| = max(0, L_b - n_sink - n_tail).
+ */
+typedef struct {
+  int32_t batch, n_q_heads, n_kv_heads, head_dim;
+  int32_t n_feat;                 /* r = d_phi */
+  int32_t n_sink, n_tail;         /* >= 0 */
+  const int64_t* cu_seqlens_host; /* host,   [batch+1], cu[0] = 0, non-decreasing */
+  const int64_t* cu_seqlens_dev;  /* device, same contents */
+  const void* k;                  /* device, bf16 */
+  const void* v;                  /* device, bf16 */
+  int64_t kv_stride_head, kv_stride_token; /* in elements */
+} tkphi_kv_desc;
+
+/* phi(x) = exp(W x + b - gamma ||x||^2); row-major fp32 parameters on the device. */
+typedef struct {
+  const float* w_q; /* [n_q_heads][n_feat][head_dim] */
+  const float* b_q; /* [n_q_heads][n_feat] */
+  const float* w_k; /* [n_kv_heads][n_feat][head_dim] */
+  const float* b_k; /* [n_kv_heads][n_feat] */
+  float gamma_q, gamma_k;
+} tkphi_phi_desc;
+
+/*
+ * Bytes of workspace the given entry point needs for this problem (0 on invalid
+ * arguments; tkphi_last_error() then says why).  topk_host (host, [batch]) may be
+ * NULL for TKPHI_WS_BUILD.  The workspace must be 256-byte aligned device memory.
+ * Its contents on entry do not matter and are undefined on exit.
+ */
+size_t tkphi_workspace_bytes(const tkphi_kv_desc* kv, const int32_t* topk_host,
+                             int32_t topk_max, int which);
+
+/*
+ * Prefill summary build (Sec. 4.1, Eq. natural_cache): for every sequence b and KV
+ * head h, S[b][h] = sum_{i in M_b} v_i phi_k(k_i)^T (row-major [head_dim][n_feat],
+ * fp32) and u[b][h] = sum_{i in M_b} phi_k(k_i) ([n_feat], fp32); both zero when the
+ * mid-region is empty.  Only phi->w_k, b_k and gamma_k are read.
+ * S: [batch][n_kv_heads][head_dim][n_feat], u: [batch][n_kv_heads][n_feat], written in full.
+ */
+tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi,
+                                   float* S, float* u,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Selection-only Top-K decode (Sec. 3, Eq. exact_terms and y_TopK = nu_E / Z_E), steps
+ * (1)-(2) above.
+ *   q         bf16 [batch][n_q_heads][head_dim], one decode query per sequence and head.
+ *   topk_host host int32 [batch]; topk_dev device copy.  0 <= topk[b] <= |M_b|
+ *             (larger is TKPHI_ERR_INVALID_ARG); topk_max >= max_b topk[b].
+ *   idx_out   int32 [batch][n_q_heads][topk_max] or NULL: the retrieved positions
+ *             within the sequence (n_sink <= i < L_b - n_tail), ascending, padded
+ *             with -1.  Equal scores are broken towards the lower index.
+ *   y_out     fp32 [batch][n_q_heads][head_dim].
+ * A sequence needs at least one anchor or one retrieved token (else INVALID_ARG).
+ */
+tkphi_status tkphi_topk_decode(const tkphi_kv_desc* kv, const void* q,
+                               const int32_t* topk_host, const int32_t* topk_dev, int32_t topk_max,
+                               int32_t* idx_out, float* y_out,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Length of one dbg_out row of tkphi_decode_step for a given head_dim. */
+#define TKPHI_DBG_STRIDE(head_dim) (4 + (head_dim))
+
+/*
+ * Top-K+phi decode step (Sec. 4.2-4.3), steps (1)-(5) above, for summaries (S, u)
+ * laid out as tkphi_build_summaries writes them.
+ *   dbg_out   fp32 [batch][n_q_heads][TKPHI_DBG_STRIDE(head_dim)] or NULL.  Per query
+ *             head: [0] m_E = max_{i in E} s_i, [1] sum_{i in E} exp(s_i - m_E),
+ *             [2] log Z_hat_R (-inf when the residual was clamped away), [3] the
+ *             common log-scale of the merge, [4..] nu_hat_R / Z_hat_R (zeros when clamped).
+ *   flags     TKPHI_FLAG_*.
+ * Clamp: a residual denominator Z_hat_R <= 0 (a finite-precision artefact of the
+ * subtraction, App. C.1) drops both residual terms, so y falls back to nu_E / Z_E.
+ * With no anchor and no retrieved token the output is nu_hat_R / Z_hat_R; if that is
+ * clamped as well the output row is zero.
+ * Other arguments as for tkphi_topk_decode.
+ */
+tkphi_status tkphi_decode_step(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, const void* q,
+                               const int32_t* topk_host, const int32_t* topk_dev, int32_t topk_max,
+                               const float* S, const float* u,
+                               int32_t* idx_out, float* y_out, float* dbg_out, uint32_t flags,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Reads the device status word that the kernels of the last call using this
+ * workspace set (0 = fine; TKPHI_ERR_TIMEOUT if a bounded wait ran out).  Waits
+ * for the stream.  *status_out is a host int.
+ */
+tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32_t* status_out);
+
+/* Message for the last error returned on the calling thread ("" if none). */
+const char* tkphi_last_error(void);
+
+/* Library version, e.g. 100 for 0.1.0. */
+int32_t tkphi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TKPHI_H */

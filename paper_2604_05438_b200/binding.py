@@ -1,0 +1,195 @@
+"""ctypes binding of libtkphi.so: same names as the C entry points, marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libtkphi.so")
+_lib = None
+
+WS_BUILD, WS_TOPK_DECODE, WS_DECODE_STEP = 0, 1, 2
+FLAG_NONE, FLAG_NOSUB = 0, 1
+
+EXPORTED_SYMBOLS = (
+    "tkphi_workspace_bytes", "tkphi_build_summaries", "tkphi_topk_decode", "tkphi_decode_step",
+    "tkphi_device_status", "tkphi_last_error", "tkphi_version",
+)
+
+
+class TkphiError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"tkphi status {status}: {message}")
+        self.status = status
+
+
+class _KvDesc(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("n_feat", C.c_int32), ("n_sink", C.c_int32),
+                ("n_tail", C.c_int32), ("cu_seqlens_host", C.c_void_p), ("cu_seqlens_dev", C.c_void_p),
+                ("k", C.c_void_p), ("v", C.c_void_p), ("kv_stride_head", C.c_int64),
+                ("kv_stride_token", C.c_int64)]
+
+
+class _PhiDesc(C.Structure):
+    _fields_ = [("w_q", C.c_void_p), ("b_q", C.c_void_p), ("w_k", C.c_void_p), ("b_k", C.c_void_p),
+                ("gamma_q", C.c_float), ("gamma_k", C.c_float)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libtkphi.so (built in-tree by ``paper_2604_05438_b200.build``); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with "
+                           "`python -m paper_2604_05438_b200.build` (there is no CPU fallback)")
+    lib = C.CDLL(_LIB_PATH)
+    lib.tkphi_workspace_bytes.restype = C.c_size_t
+    lib.tkphi_workspace_bytes.argtypes = [C.POINTER(_KvDesc), C.c_void_p, C.c_int32, C.c_int]
+    lib.tkphi_build_summaries.restype = C.c_int
+    lib.tkphi_build_summaries.argtypes = [C.POINTER(_KvDesc), C.POINTER(_PhiDesc), C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.tkphi_topk_decode.restype = C.c_int
+    lib.tkphi_topk_decode.argtypes = [C.POINTER(_KvDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.tkphi_decode_step.restype = C.c_int
+    lib.tkphi_decode_step.argtypes = [C.POINTER(_KvDesc), C.POINTER(_PhiDesc), C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.tkphi_device_status.restype = C.c_int
+    lib.tkphi_device_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+    lib.tkphi_last_error.restype = C.c_char_p
+    lib.tkphi_version.restype = C.c_int32
+    _lib = lib
+    return lib
+
+
+def _check(status: int):
+    if status != 0:
+        raise TkphiError(status, load_library().tkphi_last_error().decode())
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+@dataclass
+class KVCache:
+    """One layer's ragged K/V cache as the library sees it (no copies are made).
+
+    k, v: bf16 device tensors addressed as [head, row, dim] through the strides
+    (any layout whose innermost dim is contiguous).  cu_seqlens: int64 host array
+    [batch+1]; a device copy is kept alongside.
+    """
+    k: torch.Tensor
+    v: torch.Tensor
+    cu_seqlens: np.ndarray
+    n_q_heads: int
+    n_feat: int
+    n_sink: int
+    n_tail: int
+    cu_seqlens_dev: Optional[torch.Tensor] = None
+
+    def __post_init__(self):
+        self.cu_seqlens = np.ascontiguousarray(self.cu_seqlens, dtype=np.int64)
+        if self.cu_seqlens_dev is None:
+            self.cu_seqlens_dev = torch.from_numpy(self.cu_seqlens).to(self.k.device)
+
+    @property
+    def batch(self) -> int:
+        return len(self.cu_seqlens) - 1
+
+    def desc(self) -> _KvDesc:
+        k, v = self.k, self.v
+        assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and k.dim() == 3
+        assert k.stride() == v.stride() and k.stride(2) == 1
+        return _KvDesc(self.batch, self.n_q_heads, k.shape[0], k.shape[2], self.n_feat, self.n_sink,
+                       self.n_tail, self.cu_seqlens.ctypes.data, self.cu_seqlens_dev.data_ptr(),
+                       k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1))
+
+
+@dataclass
+class PhiMaps:
+    """fp32 device parameters of phi(x) = exp(W x + b - gamma |x|^2)."""
+    w_q: torch.Tensor
+    b_q: torch.Tensor
+    w_k: torch.Tensor
+    b_k: torch.Tensor
+    gamma_q: float
+    gamma_k: float
+
+    def desc(self) -> _PhiDesc:
+        for t in (self.w_q, self.b_q, self.w_k, self.b_k):
+            assert t.dtype == torch.float32 and t.is_contiguous()
+        return _PhiDesc(self.w_q.data_ptr(), self.b_q.data_ptr(), self.w_k.data_ptr(), self.b_k.data_ptr(),
+                        float(self.gamma_q), float(self.gamma_k))
+
+
+def _topk_host(topk) -> np.ndarray:
+    return np.ascontiguousarray(topk, dtype=np.int32)
+
+
+def workspace_bytes(kv: KVCache, topk_host, topk_max: int, which: int) -> int:
+    lib = load_library()
+    d = kv.desc()
+    th = None if topk_host is None else _topk_host(topk_host)
+    n = lib.tkphi_workspace_bytes(C.byref(d), None if th is None else th.ctypes.data, int(topk_max), which)
+    if n == 0:
+        raise TkphiError(-1, lib.tkphi_last_error().decode())
+    return int(n)
+
+
+def build_summaries(kv: KVCache, phi: PhiMaps, S: torch.Tensor, u: torch.Tensor,
+                    workspace: torch.Tensor, stream=None) -> None:
+    lib = load_library()
+    d, ph = kv.desc(), phi.desc()
+    _check(lib.tkphi_build_summaries(C.byref(d), C.byref(ph), S.data_ptr(), u.data_ptr(),
+                                     workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                     _stream_ptr(stream)))
+
+
+def topk_decode(kv: KVCache, q: torch.Tensor, topk_host, topk_dev: torch.Tensor, topk_max: int,
+                idx_out: Optional[torch.Tensor], y_out: torch.Tensor, workspace: torch.Tensor,
+                stream=None) -> None:
+    lib = load_library()
+    d = kv.desc()
+    th = _topk_host(topk_host)
+    _check(lib.tkphi_topk_decode(C.byref(d), q.data_ptr(), th.ctypes.data, topk_dev.data_ptr(), int(topk_max),
+                                 _ptr(idx_out), y_out.data_ptr(), workspace.data_ptr(),
+                                 workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
+
+
+def decode_step(kv: KVCache, phi: PhiMaps, q: torch.Tensor, topk_host, topk_dev: torch.Tensor,
+                topk_max: int, S: torch.Tensor, u: torch.Tensor, idx_out: Optional[torch.Tensor],
+                y_out: torch.Tensor, dbg_out: Optional[torch.Tensor], flags: int,
+                workspace: torch.Tensor, stream=None) -> None:
+    lib = load_library()
+    d, ph = kv.desc(), phi.desc()
+    th = _topk_host(topk_host)
+    _check(lib.tkphi_decode_step(C.byref(d), C.byref(ph), q.data_ptr(), th.ctypes.data, topk_dev.data_ptr(),
+                                 int(topk_max), S.data_ptr(), u.data_ptr(), _ptr(idx_out), y_out.data_ptr(),
+                                 _ptr(dbg_out), int(flags), workspace.data_ptr(),
+                                 workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
+
+
+def device_status(workspace: torch.Tensor, stream=None) -> int:
+    lib = load_library()
+    out = C.c_int32(0)
+    _check(lib.tkphi_device_status(workspace.data_ptr(), _stream_ptr(stream), C.byref(out)))
+    return int(out.value)

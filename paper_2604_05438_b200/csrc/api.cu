@@ -1,0 +1,356 @@
+// C ABI of libtkphi: argument validation, workspace layout, launches.
+#include "../../include/tkphi.h"
+#include "common.cuh"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+using namespace tkphi;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+tkphi_status fail(tkphi_status st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Shape {
+  long long total_tokens;
+  int max_len, max_mid, rows, units;
+  long long score_tiles;          // tiles of the scoring kernel (all units)
+};
+
+tkphi_status validate_kv(const tkphi_kv_desc* kv, Shape* sh, bool need_data) {
+  if (!kv) return fail(TKPHI_ERR_INVALID_ARG, "kv descriptor is NULL");
+  if (kv->batch < 1 || kv->batch > kMaxBatch)
+    return fail(TKPHI_ERR_INVALID_ARG, "batch must be in [1, %d], got %d", kMaxBatch, kv->batch);
+  if (kv->head_dim != 64 && kv->head_dim != 128)
+    return fail(TKPHI_ERR_UNSUPPORTED, "head_dim must be 64 or 128, got %d", kv->head_dim);
+  if (kv->n_feat != 64 && kv->n_feat != 128)
+    return fail(TKPHI_ERR_UNSUPPORTED, "n_feat must be 64 or 128, got %d", kv->n_feat);
+  if (kv->n_kv_heads < 1 || kv->n_q_heads < 1 || kv->n_q_heads % kv->n_kv_heads != 0)
+    return fail(TKPHI_ERR_INVALID_ARG, "n_q_heads (%d) must be a positive multiple of n_kv_heads (%d)",
+                kv->n_q_heads, kv->n_kv_heads);
+  if (kv->n_q_heads / kv->n_kv_heads > 8)
+    return fail(TKPHI_ERR_UNSUPPORTED, "group size %d > 8", kv->n_q_heads / kv->n_kv_heads);
+  if (kv->n_sink < 0 || kv->n_tail < 0) return fail(TKPHI_ERR_INVALID_ARG, "negative anchor count");
+  if (!kv->cu_seqlens_host) return fail(TKPHI_ERR_INVALID_ARG, "cu_seqlens_host is NULL");
+  const int64_t* cu = kv->cu_seqlens_host;
+  if (cu[0] != 0) return fail(TKPHI_ERR_INVALID_ARG, "cu_seqlens[0] must be 0");
+  sh->max_len = 0; sh->max_mid = 0;
+  for (int b = 0; b < kv->batch; ++b) {
+    const int64_t len = cu[b + 1] - cu[b];
+    if (len < 1) return fail(TKPHI_ERR_INVALID_ARG, "sequence %d has length %lld (< 1)", b, (long long)len);
+    if (cu[b + 1] >= (1ll << 31)) return fail(TKPHI_ERR_INVALID_ARG, "more than 2^31-1 cache rows");
+    if (len > sh->max_len) sh->max_len = (int)len;
+    const int64_t mid = len - kv->n_sink - kv->n_tail;
+    if (mid > sh->max_mid) sh->max_mid = (int)mid;
+  }
+  sh->total_tokens = cu[kv->batch];
+  sh->rows = kv->batch * kv->n_q_heads;
+  sh->units = kv->batch * kv->n_kv_heads;
+  if (need_data) {
+    if (!kv->cu_seqlens_dev) return fail(TKPHI_ERR_INVALID_ARG, "cu_seqlens_dev is NULL");
+    if (!kv->k || !kv->v) return fail(TKPHI_ERR_INVALID_ARG, "k or v is NULL");
+    if (!aligned16(kv->k) || !aligned16(kv->v)) return fail(TKPHI_ERR_INVALID_ARG, "k and v must be 16-byte aligned");
+    if (kv->kv_stride_token < kv->head_dim || kv->kv_stride_token % 8 != 0 || kv->kv_stride_head % 8 != 0 ||
+        kv->kv_stride_head < 0)
+      return fail(TKPHI_ERR_INVALID_ARG, "strides must be multiples of 8 elements, token stride >= head_dim");
+  }
+  return TKPHI_OK;
+}
+
+tkphi_status validate_topk(const tkphi_kv_desc* kv, const int32_t* topk_host, int32_t topk_max, Shape* sh,
+                           bool allow_empty_support) {
+  if (!topk_host) return fail(TKPHI_ERR_INVALID_ARG, "topk_host is NULL");
+  if (topk_max < 0) return fail(TKPHI_ERR_INVALID_ARG, "topk_max < 0");
+  const int64_t* cu = kv->cu_seqlens_host;
+  const int tk = score_tile_keys(kv->head_dim);
+  sh->score_tiles = 0;
+  for (int b = 0; b < kv->batch; ++b) {
+    const int64_t len = cu[b + 1] - cu[b];
+    int64_t mid = len - kv->n_sink - kv->n_tail;
+    if (mid < 0) mid = 0;
+    if (topk_host[b] < 0 || topk_host[b] > mid)
+      return fail(TKPHI_ERR_INVALID_ARG, "topk[%d] = %d outside [0, |M| = %lld]", b, topk_host[b], (long long)mid);
+    if (topk_host[b] > topk_max)
+      return fail(TKPHI_ERR_INVALID_ARG, "topk[%d] = %d exceeds topk_max = %d", b, topk_host[b], topk_max);
+    if (!allow_empty_support && topk_host[b] == 0 && kv->n_sink == 0 && kv->n_tail == 0)
+      return fail(TKPHI_ERR_INVALID_ARG, "sequence %d has an empty exact support (no anchors, topk = 0)", b);
+    if (topk_host[b] > 0) sh->score_tiles += (int64_t)kv->n_kv_heads * ((mid + tk - 1) / tk);
+  }
+  if (sh->score_tiles >= (1ll << 31)) return fail(TKPHI_ERR_UNSUPPORTED, "too many key tiles");
+  return TKPHI_OK;
+}
+
+int n_sm_cached() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, WsLayout* L) {
+  const int passes = (kv->n_q_heads / kv->n_kv_heads + 3) / 4;
+  size_t o = 0;
+  L->passes = passes;
+  L->status = o;        o += 256;
+  L->unit_counter = o;  o = align_up(o + sizeof(unsigned) * sh.units * passes, 256);
+  L->row_counter = o;   o = align_up(o + sizeof(unsigned) * sh.rows, 256);
+  L->hist = o;          o = align_up(o + sizeof(unsigned) * (size_t)sh.rows * kHistBins, 256);
+  L->zero_end = o;
+  L->rowinfo = o;       o = align_up(o + sizeof(int4) * sh.rows, 256);
+  L->scores = o;        o = align_up(o + sizeof(float) * (size_t)kv->n_q_heads * sh.total_tokens, 256);
+  const size_t bm_words = ((size_t)kv->n_q_heads * sh.total_tokens) / 32 + sh.rows + 2;
+  L->bm_sure = o;       o = align_up(o + 4 * bm_words, 256);
+  L->bm_cand = o;       o = align_up(o + 4 * bm_words, 256);
+  L->idx = o;           o = align_up(o + sizeof(int) * (size_t)sh.rows * (topk_max > 0 ? topk_max : 1), 256);
+  L->aq = o;            o = align_up(o + sizeof(float) * (size_t)sh.rows * (kv->n_feat + 4), 256);
+  int64_t max_support = (int64_t)kv->n_sink + kv->n_tail + topk_max;
+  if (max_support > sh.max_len) max_support = sh.max_len;
+  L->max_slices = (int)((max_support + kSlice - 1) / kSlice);
+  if (L->max_slices < 1) L->max_slices = 1;
+  L->partial_stride = 4 + 2 * kv->head_dim;
+  L->partials = o;      o = align_up(o + sizeof(float) * (size_t)sh.rows * L->max_slices * L->partial_stride, 256);
+  L->total = o;
+}
+
+void build_layout(const tkphi_kv_desc* kv, const Shape& sh, WsLayout* L) {
+  size_t o = 0;
+  L->status = o;        o += 256;
+  L->unit_counter = o;  o = align_up(o + sizeof(unsigned) * sh.units, 256);
+  L->zero_end = o;
+  // about two CTAs per SM over all units, at least 2048 mid tokens per CTA
+  const int64_t total_mid = (int64_t)sh.max_mid > 0 ? (int64_t)sh.max_mid * sh.units : 0;
+  int64_t chunk = (total_mid + 2 * 148 - 1) / (2 * 148);
+  if (chunk < 2048) chunk = 2048;
+  chunk = (chunk + 31) / 32 * 32;
+  L->chunk_len = (int)chunk;
+  L->chunks_per_unit = sh.max_mid > 0 ? (int)((sh.max_mid + chunk - 1) / chunk) : 1;
+  L->b_partials = o;
+  o = align_up(o + sizeof(float) * (size_t)sh.units * L->chunks_per_unit *
+                       ((size_t)kv->head_dim * kv->n_feat + kv->n_feat), 256);
+  L->total = o;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// 3-D view [head][row][dim] of the key cache; box = one scoring tile of one head.
+tkphi_status make_key_tensor_map(const tkphi_kv_desc* kv, long long total_tokens, CUtensorMap* tm) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return fail(TKPHI_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  const cuuint64_t dims[3] = {(cuuint64_t)kv->head_dim, (cuuint64_t)total_tokens, (cuuint64_t)kv->n_kv_heads};
+  const cuuint64_t strides[2] = {(cuuint64_t)kv->kv_stride_token * 2, (cuuint64_t)kv->kv_stride_head * 2};
+  const cuuint32_t box[3] = {(cuuint32_t)kv->head_dim, (cuuint32_t)score_tile_keys(kv->head_dim), 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  // a single head (stride 0 would be rejected): give the unused dimension a legal stride
+  cuuint64_t st[2] = {strides[0], strides[1]};
+  if (kv->n_kv_heads == 1 || st[1] == 0) st[1] = st[0] * (cuuint64_t)total_tokens;
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(kv->k), dims, st, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(TKPHI_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return TKPHI_OK;
+}
+
+tkphi_status check_ws(void* ws, size_t have, size_t need) {
+  if (!ws) return fail(TKPHI_ERR_WORKSPACE, "workspace is NULL");
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(TKPHI_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+  if (have < need) return fail(TKPHI_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", have, need);
+  return TKPHI_OK;
+}
+
+tkphi_status cuda_fail(cudaError_t e, const char* what) {
+  return fail(TKPHI_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, const void* q,
+                           const int32_t* topk_host, const int32_t* topk_dev, int32_t topk_max, const float* S,
+                           const float* u, int32_t* idx_out, float* y_out, float* dbg_out, uint32_t flags,
+                           void* ws, size_t ws_bytes, void* stream, bool with_phi) {
+  g_err[0] = 0;
+  Shape sh{};
+  tkphi_status st = validate_kv(kv, &sh, true);
+  if (st != TKPHI_OK) return st;
+  st = validate_topk(kv, topk_host, topk_max, &sh, with_phi);
+  if (st != TKPHI_OK) return st;
+  if (!topk_dev) return fail(TKPHI_ERR_INVALID_ARG, "topk_dev is NULL");
+  if (!q || !aligned16(q)) return fail(TKPHI_ERR_INVALID_ARG, "q is NULL or not 16-byte aligned");
+  if (!y_out) return fail(TKPHI_ERR_INVALID_ARG, "y_out is NULL");
+  if (flags & ~1u) return fail(TKPHI_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
+  if (with_phi) {
+    if (!phi || !phi->w_q || !phi->b_q || !phi->w_k || !phi->b_k)
+      return fail(TKPHI_ERR_INVALID_ARG, "phi descriptor or one of its pointers is NULL");
+    if (!S || !u) return fail(TKPHI_ERR_INVALID_ARG, "S or u is NULL");
+    if (!std::isfinite(phi->gamma_q) || !std::isfinite(phi->gamma_k))
+      return fail(TKPHI_ERR_INVALID_ARG, "gamma must be finite");
+  }
+  WsLayout L{};
+  decode_layout(kv, sh, topk_max, &L);
+  st = check_ws(ws, ws_bytes, L.total);
+  if (st != TKPHI_OK) return st;
+
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  Problem p{};
+  p.batch = kv->batch; p.n_q_heads = kv->n_q_heads; p.n_kv_heads = kv->n_kv_heads;
+  p.head_dim = kv->head_dim; p.n_feat = kv->n_feat; p.n_sink = kv->n_sink; p.n_tail = kv->n_tail;
+  p.group = kv->n_q_heads / kv->n_kv_heads;
+  p.cu_seqlens = reinterpret_cast<const long long*>(kv->cu_seqlens_dev);
+  p.topk = topk_dev; p.topk_max = topk_max > 0 ? topk_max : 1;
+  p.k = static_cast<const __nv_bfloat16*>(kv->k); p.v = static_cast<const __nv_bfloat16*>(kv->v);
+  p.stride_head = kv->kv_stride_head; p.stride_token = kv->kv_stride_token;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  if (with_phi) {
+    p.w_q = phi->w_q; p.b_q = phi->b_q; p.w_k = phi->w_k; p.b_k = phi->b_k;
+    p.gamma_q = phi->gamma_q; p.gamma_k = phi->gamma_k; p.S = S; p.u = u;
+  }
+  p.idx_out = idx_out; p.y_out = y_out; p.dbg_out = dbg_out; p.flags = flags; p.with_phi = with_phi ? 1 : 0;
+  p.status = reinterpret_cast<int*>(w + L.status);
+  p.unit_counter = reinterpret_cast<unsigned*>(w + L.unit_counter);
+  p.row_counter = reinterpret_cast<unsigned*>(w + L.row_counter);
+  p.rowinfo = reinterpret_cast<int4*>(w + L.rowinfo);
+  p.hist = reinterpret_cast<unsigned*>(w + L.hist);
+  p.scores = reinterpret_cast<float*>(w + L.scores);
+  p.bm_sure = reinterpret_cast<unsigned*>(w + L.bm_sure);
+  p.bm_cand = reinterpret_cast<unsigned*>(w + L.bm_cand);
+  p.idx = reinterpret_cast<int*>(w + L.idx);
+  p.aq = reinterpret_cast<float*>(w + L.aq);
+  p.partials = reinterpret_cast<float*>(w + L.partials);
+  p.max_slices = L.max_slices; p.partial_stride = L.partial_stride;
+  p.scale = 1.0f / sqrtf((float)kv->head_dim);
+  // idx_out uses the caller's topk_max as its row length; the internal list uses p.topk_max
+  if (topk_max == 0) p.idx_out = nullptr;
+
+  cudaError_t e = cudaMemsetAsync(w, 0, L.zero_end, cs);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
+  if (sh.score_tiles > 0) {
+    CUtensorMap tm;
+    st = make_key_tensor_map(kv, sh.total_tokens, &tm);
+    if (st != TKPHI_OK) return st;
+    long long grid = sh.score_tiles < n_sm_cached() ? sh.score_tiles : n_sm_cached();
+    for (int pass = 0; pass < L.passes; ++pass) {
+      e = launch_score_hist(p, tm, pass, (int)grid, cs);
+      if (e != cudaSuccess) return cuda_fail(e, "score_hist launch");
+    }
+    e = launch_partition(p, sh.max_mid, cs);
+    if (e != cudaSuccess) return cuda_fail(e, "partition launch");
+  }
+  e = launch_finalize_select(p, cs);
+  if (e != cudaSuccess) return cuda_fail(e, "finalize_select launch");
+  e = launch_exact_residual(p, cs);
+  if (e != cudaSuccess) return cuda_fail(e, "exact_residual launch");
+  return TKPHI_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* tkphi_last_error(void) { return g_err; }
+int32_t tkphi_version(void) { return 100; }
+
+size_t tkphi_workspace_bytes(const tkphi_kv_desc* kv, const int32_t* topk_host, int32_t topk_max, int which) {
+  g_err[0] = 0;
+  Shape sh{};
+  if (validate_kv(kv, &sh, false) != TKPHI_OK) return 0;
+  WsLayout L{};
+  if (which == TKPHI_WS_BUILD) {
+    build_layout(kv, sh, &L);
+    return L.total;
+  }
+  if (which != TKPHI_WS_TOPK_DECODE && which != TKPHI_WS_DECODE_STEP) {
+    fail(TKPHI_ERR_INVALID_ARG, "unknown workspace kind %d", which);
+    return 0;
+  }
+  if (validate_topk(kv, topk_host, topk_max, &sh, true) != TKPHI_OK) return 0;
+  decode_layout(kv, sh, topk_max, &L);
+  return L.total;
+}
+
+tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, float* S, float* u,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  g_err[0] = 0;
+  Shape sh{};
+  tkphi_status st = validate_kv(kv, &sh, true);
+  if (st != TKPHI_OK) return st;
+  if (!phi || !phi->w_k || !phi->b_k) return fail(TKPHI_ERR_INVALID_ARG, "phi->w_k or phi->b_k is NULL");
+  if (!std::isfinite(phi->gamma_k)) return fail(TKPHI_ERR_INVALID_ARG, "gamma_k must be finite");
+  if (!S || !u) return fail(TKPHI_ERR_INVALID_ARG, "S or u is NULL");
+  WsLayout L{};
+  build_layout(kv, sh, &L);
+  st = check_ws(workspace, workspace_bytes, L.total);
+  if (st != TKPHI_OK) return st;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* w = static_cast<char*>(workspace);
+  BuildProblem p{};
+  p.batch = kv->batch; p.n_kv_heads = kv->n_kv_heads; p.head_dim = kv->head_dim; p.n_feat = kv->n_feat;
+  p.n_sink = kv->n_sink; p.n_tail = kv->n_tail;
+  p.cu_seqlens = reinterpret_cast<const long long*>(kv->cu_seqlens_dev);
+  p.k = static_cast<const __nv_bfloat16*>(kv->k); p.v = static_cast<const __nv_bfloat16*>(kv->v);
+  p.stride_head = kv->kv_stride_head; p.stride_token = kv->kv_stride_token;
+  p.w_k = phi->w_k; p.b_k = phi->b_k; p.gamma_k = phi->gamma_k;
+  p.S = S; p.u = u;
+  p.status = reinterpret_cast<int*>(w + L.status);
+  p.unit_counter = reinterpret_cast<unsigned*>(w + L.unit_counter);
+  p.partials = reinterpret_cast<float*>(w + L.b_partials);
+  p.chunk_len = L.chunk_len; p.chunks_per_unit = L.chunks_per_unit;
+  cudaError_t e = cudaMemsetAsync(w, 0, L.zero_end, cs);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
+  e = launch_build(p, cs);
+  if (e != cudaSuccess) return cuda_fail(e, "build launch");
+  return TKPHI_OK;
+}
+
+tkphi_status tkphi_topk_decode(const tkphi_kv_desc* kv, const void* q, const int32_t* topk_host,
+                               const int32_t* topk_dev, int32_t topk_max, int32_t* idx_out, float* y_out,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return decode_common(kv, nullptr, q, topk_host, topk_dev, topk_max, nullptr, nullptr, idx_out, y_out, nullptr, 0,
+                       workspace, workspace_bytes, cuda_stream, false);
+}
+
+tkphi_status tkphi_decode_step(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, const void* q,
+                               const int32_t* topk_host, const int32_t* topk_dev, int32_t topk_max, const float* S,
+                               const float* u, int32_t* idx_out, float* y_out, float* dbg_out, uint32_t flags,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return decode_common(kv, phi, q, topk_host, topk_dev, topk_max, S, u, idx_out, y_out, dbg_out, flags, workspace,
+                       workspace_bytes, cuda_stream, true);
+}
+
+tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32_t* status_out) {
+  g_err[0] = 0;
+  if (!workspace || !status_out) return fail(TKPHI_ERR_INVALID_ARG, "NULL argument");
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(status_out, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, cs);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
+  if (e != cudaSuccess) return cuda_fail(e, "reading the device status word");
+  return TKPHI_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,167 @@
+// Shared declarations of the libtkphi kernels: problem description, workspace
+// layout, small device helpers.  sm_100a only.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <stddef.h>
+
+namespace tkphi {
+
+constexpr int kHistBits = 12;                 // leading bits of the ordered score key
+constexpr int kHistBins = 1 << kHistBits;     // bins of the fused first-pass histogram
+constexpr int kLowBits = 32 - kHistBits;      // bits refined inside the threshold bin
+constexpr int kMaxBatch = 4096;               // sequences per call
+constexpr int kSlice = 64;                    // exact-support tokens per CTA of the exact/residual kernel
+constexpr uint32_t kSpinLimit = 1u << 22;     // polls of a bounded mbarrier wait (with back-off)
+
+// Device status word values (first word of the workspace).
+constexpr int kStatusOk = 0;
+constexpr int kStatusTimeout = -5;
+
+// Everything the kernels need to know about one layer call.
+struct Problem {
+  int batch, n_q_heads, n_kv_heads, head_dim, n_feat, n_sink, n_tail, group;
+  const long long* cu_seqlens;     // device [batch+1]
+  const int* topk;                 // device [batch] (null for the build)
+  int topk_max;
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  long long stride_head, stride_token;   // elements
+  const __nv_bfloat16* q;          // [batch][n_q_heads][head_dim]
+  // feature maps
+  const float* w_q; const float* b_q; const float* w_k; const float* b_k;
+  float gamma_q, gamma_k;
+  // summaries
+  const float* S; const float* u;
+  // outputs
+  int* idx_out; float* y_out; float* dbg_out;
+  unsigned flags;
+  int with_phi;                    // 0: selection-only, 1: Top-K+phi
+  // workspace pieces (device pointers)
+  int* status;
+  unsigned* unit_counter;          // [batch*n_kv_heads*passes]
+  unsigned* row_counter;           // [batch*n_q_heads]
+  int4* rowinfo;                   // [rows]: x = threshold bin, y = count above, z = count in bin
+  unsigned* hist;                  // [rows][kHistBins]
+  float* scores;                   // [n_q_heads * total_tokens]
+  unsigned* bm_sure;               // bitmap of surely selected mid positions
+  unsigned* bm_cand;               // bitmap of threshold-bin candidates
+  int* idx;                        // [rows][topk_max] ascending retrieved positions
+  float* aq;                       // [rows][n_feat + 4]: exp(a_q - m_q) per feature, then m_q
+  float* partials;                 // [rows][max_slices][partial_stride]
+  int max_slices, partial_stride;
+  float scale;                     // 1/sqrt(head_dim)
+};
+
+struct BuildProblem {
+  int batch, n_kv_heads, head_dim, n_feat, n_sink, n_tail;
+  const long long* cu_seqlens;
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  long long stride_head, stride_token;
+  const float* w_k; const float* b_k; float gamma_k;
+  float* S; float* u;
+  int* status;
+  unsigned* unit_counter;          // [batch*n_kv_heads]
+  float* partials;                 // [units][chunks_per_unit][d*r + r]
+  int chunk_len;                   // mid tokens per CTA
+  int chunks_per_unit;             // upper bound over sequences
+};
+
+// Host-side byte offsets of the workspace pieces.
+struct WsLayout {
+  size_t status, unit_counter, row_counter, hist, zero_end;
+  size_t rowinfo, scores, bm_sure, bm_cand, idx, aq, partials, total;
+  int max_slices, partial_stride, passes;
+  // build
+  size_t b_partials; int chunk_len, chunks_per_unit;
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// keys per TMA tile of the scoring kernel (32 KB of bf16 rows)
+__host__ __device__ inline int score_tile_keys(int head_dim) { return head_dim == 64 ? 256 : 128; }
+
+// ---------------------------------------------------------------- device helpers
+__device__ __forceinline__ int mid_len(long long n, int n_sink, int n_tail) {
+  long long m = n - n_sink - n_tail;
+  return m > 0 ? (int)m : 0;
+}
+
+// Order-preserving map from fp32 to uint32: larger float <=> larger key.
+__device__ __forceinline__ unsigned ordered_key(float f) {
+  unsigned u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float bf16_lo(unsigned packed) { return __uint_as_float(packed << 16); }
+__device__ __forceinline__ float bf16_hi(unsigned packed) { return __uint_as_float(packed & 0xffff0000u); }
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+__device__ __forceinline__ int warp_sum_int(int x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+// Exclusive prefix sum of one int per thread over the block; returns the
+// exclusive prefix, *total gets the block sum.  `scratch` holds >= 33 ints.
+// All threads of the block must call it; blockDim.x is a multiple of 32, <= 1024.
+__device__ __forceinline__ int block_exclusive_scan(int x, int* scratch, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  int incl = x;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  __syncthreads();                     // scratch may still be in use by a previous scan
+  if (lane == 31) scratch[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = lane < nwarp ? scratch[lane] : 0;
+    int wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += y;
+    }
+    scratch[lane] = wi - w;            // exclusive prefix of warp sums
+    if (lane == 31) scratch[32] = wi;
+  }
+  __syncthreads();
+  int res = scratch[warp] + incl - x;
+  *total = scratch[32];
+  return res;
+}
+
+// Offsets that follow from cu_seqlens alone (no per-call prefix arrays needed):
+// the score row of (b, hq) starts at element H_q*cu[b] + hq*L_b, and its bitmap
+// at word (that offset)/32 + row, which never overlaps the next row's words.
+__device__ __forceinline__ long long score_row_base(const Problem& p, int b, int hq, long long cu_b, long long len_b) {
+  return (long long)p.n_q_heads * cu_b + (long long)hq * len_b;
+}
+__device__ __forceinline__ long long bitmap_row_base(const Problem& p, int b, int hq, long long cu_b, long long len_b) {
+  return (score_row_base(p, b, hq, cu_b, len_b) >> 5) + (long long)(b * p.n_q_heads + hq);
+}
+
+// ---------------------------------------------------------------- host launchers
+// Each returns cudaGetLastError() after enqueuing on `stream`.
+cudaError_t launch_score_hist(const Problem& p, const CUtensorMap& tmap_k, int pass, int n_sm, cudaStream_t stream);
+cudaError_t launch_partition(const Problem& p, int max_mid, cudaStream_t stream);
+cudaError_t launch_finalize_select(const Problem& p, cudaStream_t stream);
+cudaError_t launch_exact_residual(const Problem& p, cudaStream_t stream);
+cudaError_t launch_build(const BuildProblem& p, cudaStream_t stream);
+
+}  // namespace tkphi

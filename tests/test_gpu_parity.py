@@ -1,0 +1,248 @@
+"""CUDA path vs float64 oracle, element by element, through the C ABI.  Needs a GPU."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import tkphi_oracle as O
+from workloads import CONFIGS, make_layer_inputs, make_phi_params
+
+import parity_utils as PU
+
+pytestmark = pytest.mark.gpu
+
+
+def _cfg(name, **kw):
+    return dataclasses.replace(CONFIGS[name], **kw)
+
+
+def _phi_arrays(phi, hq, kvh):
+    return (phi.w_q[hq].double().numpy(), phi.b_q[hq].double().numpy(), phi.gamma_q,
+            phi.w_k[kvh].double().numpy(), phi.b_k[kvh].double().numpy(), phi.gamma_k)
+
+
+def _check_build(gl, S, u, heads=None):
+    cfg, inp, phi = gl.cfg, gl.inp, gl.phi
+    Sh, uh = S.cpu().numpy(), u.cpu().numpy()
+    assert np.isfinite(Sh).all() and np.isfinite(uh).all()
+    worst = 0.0
+    for b in range(inp.batch):
+        for kvh in (range(cfg.n_kv_heads) if heads is None else heads):
+            K, V = PU.seq_arrays(inp, b, kvh)
+            S0, u0 = O.build_summaries(K, V, phi.w_k[kvh].double().numpy(), phi.b_k[kvh].double().numpy(),
+                                       phi.gamma_k, inp.n_sink, inp.n_tail)
+            if np.abs(S0).max() == 0:
+                assert np.abs(Sh[b, kvh]).max() == 0 and np.abs(uh[b, kvh]).max() == 0
+                continue
+            eS, eu = PU.max_rel(Sh[b, kvh], S0), PU.max_rel(uh[b, kvh], u0)
+            worst = max(worst, eS, eu)
+            assert eS <= PU.SU_TOL and eu <= PU.SU_TOL, (b, kvh, eS, eu)
+    return worst
+
+
+def _check_decode(gl, step, frac, S, u, with_phi=True, flags=0, heads=None, topk=None, topk_max=None,
+                  check_resid=True):
+    cfg, inp, phi = gl.cfg, gl.inp, gl.phi
+    topk = inp.topk(frac) if topk is None else np.asarray(topk, np.int32)
+    q = inp.q[step]
+    out = PU.gpu_decode(gl, q, topk, S, u, with_phi=with_phi, flags=flags, topk_max=topk_max)
+    Sh = None if S is None else S.cpu().double().numpy()
+    uh = None if u is None else u.cpu().double().numpy()
+    G = cfg.group
+    worst = 0.0
+    for b in range(inp.batch):
+        for hq in (range(cfg.n_q_heads) if heads is None else heads):
+            kvh = hq // G
+            K, V = PU.seq_arrays(inp, b, kvh)
+            q64 = q[b, hq].double().numpy()
+            kk = int(topk[b])
+            if out["idx"] is not None and (topk_max or topk.max()) > 0:
+                ret = PU.check_selection(q64, K, inp.n_sink, inp.n_tail, kk, out["idx"][b, hq])
+            else:
+                ret = O.select_topk(q64, K, inp.n_sink, inp.n_tail, kk)
+            if with_phi:
+                res = O.topkphi_attention(q64, K, V, inp.n_sink, inp.n_tail, kk, *_phi_arrays(phi, hq, kvh),
+                                          S=Sh[b, kvh], u=uh[b, kvh], retrieved=ret,
+                                          subtract=not (flags & 1))
+                y0 = res.y
+                dbg = out["dbg"][b, hq]
+                if math.isfinite(res.m_E):
+                    assert abs(dbg[0] - res.m_E) <= PU.ME_TOL * max(1.0, abs(res.m_E)), (b, hq, dbg[0], res.m_E)
+                    assert abs(dbg[1] - res.Z_E) <= 1e-4 * res.Z_E
+                if check_resid and not res.clamped and math.isfinite(dbg[2]):
+                    assert abs(dbg[2] - res.log_Zhat_R) <= PU.LOGZ_TOL, (b, hq, dbg[2], res.log_Zhat_R)
+                    assert PU.max_rel(dbg[4:], res.y_R_hat) <= PU.Y_TOL, (b, hq)
+            else:
+                y0, _ = O.topk_attention(q64, K, V, inp.n_sink, inp.n_tail, kk, retrieved=ret)
+            e = PU.max_rel(out["y"][b, hq], y0)
+            worst = max(worst, e)
+            assert e <= PU.Y_TOL, (b, hq, e)
+    return worst
+
+
+# ------------------------------------------------------------------ config 1, full size
+@pytest.mark.parametrize("seed", [0, 1])
+def test_c1_full_size_topk_and_topkphi(seed):
+    cfg = CONFIGS["c1_1b_4k"]
+    inp = make_layer_inputs(cfg, seed, n_steps=3)
+    phi = make_phi_params(cfg, seed)
+    gl = PU.to_gpu(cfg, inp, phi)
+    S, u = PU.gpu_build(gl)
+    _check_build(gl, S, u)
+    for step in range(3):
+        _check_decode(gl, step, 0.01, None, None, with_phi=False)
+        _check_decode(gl, step, 0.01, S, u, with_phi=True)
+
+
+def test_c1_visible_residual_phi():
+    cfg = CONFIGS["c1_1b_4k"]
+    inp = make_layer_inputs(cfg, 2, n_steps=2)
+    phi0 = make_phi_params(cfg, 2, kind="visible")
+    shift = PU.calibrate_visible_shift(cfg, inp, phi0, 0.01)
+    phi = make_phi_params(cfg, 2, kind="visible", bk_shift=shift)
+    gl = PU.to_gpu(cfg, inp, phi)
+    S, u = PU.gpu_build(gl)
+    _check_build(gl, S, u)
+    for step in range(2):
+        _check_decode(gl, step, 0.01, S, u)
+        _check_decode(gl, step, 0.01, S, u, flags=1)          # NoSub ablation
+    # the residual must actually matter here: Top-K+phi differs visibly from Top-K
+    out_phi = PU.gpu_decode(gl, inp.q[0], inp.topk(0.01), S, u)
+    out_top = PU.gpu_decode(gl, inp.q[0], inp.topk(0.01), with_phi=False)
+    assert np.abs(out_phi["y"] - out_top["y"]).max() > 1e-2
+
+
+# ------------------------------------------------------------------ 3B geometry, several tiles + ragged tail
+@pytest.mark.parametrize("kind", ["baseline", "visible"])
+def test_c3_geometry_reduced_length(kind):
+    cfg = _cfg("c3_3b_128k", needle_every=512)
+    inp = make_layer_inputs(cfg, 0, seq_lens=[5000], n_steps=2)
+    phi = make_phi_params(cfg, 0, kind=kind)
+    if kind == "visible":
+        phi = make_phi_params(cfg, 0, kind=kind, bk_shift=PU.calibrate_visible_shift(cfg, inp, phi, 0.02))
+    gl = PU.to_gpu(cfg, inp, phi)
+    S, u = PU.gpu_build(gl)
+    _check_build(gl, S, u)
+    for frac in (0.005, 0.04):
+        _check_decode(gl, 0, frac, S, u)
+    _check_decode(gl, 1, 0.02, None, None, with_phi=False)
+
+
+# ------------------------------------------------------------------ ragged batch (config 4 shape, small lengths)
+def test_c4_ragged_batch():
+    cfg = _cfg("c4_1b_ragged", batch=5)
+    inp = make_layer_inputs(cfg, 3, seq_lens=[700, 69, 2049, 68, 1300], n_steps=1)
+    phi = make_phi_params(cfg, 3)
+    gl = PU.to_gpu(cfg, inp, phi)
+    S, u = PU.gpu_build(gl)
+    _check_build(gl, S, u)
+    topk = inp.topk(0.05)
+    assert topk.tolist()[1] == 0 and topk.tolist()[3] == 0
+    _check_decode(gl, 0, 0.05, S, u, topk=topk, topk_max=int(topk.max()) + 5)
+    _check_decode(gl, 0, 0.05, None, None, with_phi=False, topk=topk)
+
+
+def test_c5_zipf_norms_reduced_length():
+    cfg = _cfg("c5_3b_1m", batch=2)
+    inp = make_layer_inputs(cfg, 1, seq_lens=[6000, 3001], n_steps=1)
+    phi = make_phi_params(cfg, 1)
+    gl = PU.to_gpu(cfg, inp, phi)
+    S, u = PU.gpu_build(gl)
+    _check_build(gl, S, u)
+    _check_decode(gl, 0, 0.01, S, u, heads=range(0, 24, 5))
+
+
+# ------------------------------------------------------------------ layouts and head groupings
+def test_token_major_layout_and_group_of_eight():
+    cfg = _cfg("c1_1b_4k", n_q_heads=16, n_kv_heads=2)        # G = 8: two scoring passes
+    inp = make_layer_inputs(cfg, 5, seq_lens=[1500], n_steps=1)
+    phi = make_phi_params(cfg, 5)
+    gl = PU.to_gpu(cfg, inp, phi, token_major=True)
+    S, u = PU.gpu_build(gl)
+    _check_build(gl, S, u)
+    _check_decode(gl, 0, 0.03, S, u)
+
+
+def test_mixed_dims_d64_r128_and_d128_r64():
+    for d, r in ((64, 128), (128, 64)):
+        cfg = _cfg("c1_1b_4k", head_dim=d, n_feat=r, n_q_heads=6, n_kv_heads=2)   # G = 3
+        inp = make_layer_inputs(cfg, 6, seq_lens=[900], n_steps=1)
+        phi = make_phi_params(cfg, 6)
+        gl = PU.to_gpu(cfg, inp, phi)
+        S, u = PU.gpu_build(gl)
+        _check_build(gl, S, u)
+        _check_decode(gl, 0, 0.02, S, u)
+
+
+# ------------------------------------------------------------------ degenerate cases
+def test_budget_edges_zero_and_full():
+    cfg = _cfg("c1_1b_4k", n_q_heads=8, n_kv_heads=2)
+    inp = make_layer_inputs(cfg, 7, seq_lens=[600], n_steps=1)
+    phi0 = make_phi_params(cfg, 7, kind="visible")
+    phi = make_phi_params(cfg, 7, kind="visible", bk_shift=PU.calibrate_visible_shift(cfg, inp, phi0, 0.05))
+    gl = PU.to_gpu(cfg, inp, phi)
+    S, u = PU.gpu_build(gl)
+    n_mid = 600 - 68
+    # K = 0: anchors plus the whole-mid residual
+    _check_decode(gl, 0, 0.0, S, u, topk=[0])
+    _check_decode(gl, 0, 0.0, None, None, with_phi=False, topk=[0])
+    # K = 1 and K = |M| - 1
+    _check_decode(gl, 0, 0.0, S, u, topk=[1])
+    _check_decode(gl, 0, 0.0, S, u, topk=[n_mid - 1], check_resid=False)
+    # K = |M|: residual summaries cancel -> full attention (invariant of the method)
+    out = PU.gpu_decode(gl, inp.q[0], np.array([n_mid], np.int32), S, u)
+    assert (out["idx"][0, :, :n_mid] == np.arange(4, 600 - 64)).all()
+    for hq in range(cfg.n_q_heads):
+        K, V = PU.seq_arrays(inp, 0, hq // cfg.group)
+        y_full = O.full_attention(inp.q[0, 0, hq].double().numpy(), K, V)
+        assert PU.max_rel(out["y"][0, hq], y_full) <= PU.Y_TOL
+
+
+def test_no_anchors_and_tiny_sequences():
+    cfg = _cfg("c1_1b_4k", n_q_heads=4, n_kv_heads=1, n_sink=0, n_tail=0)
+    inp = make_layer_inputs(cfg, 8, seq_lens=[1, 257, 33], n_steps=1)
+    phi = make_phi_params(cfg, 8)
+    gl = PU.to_gpu(cfg, inp, phi)
+    S, u = PU.gpu_build(gl)
+    _check_build(gl, S, u)
+    _check_decode(gl, 0, 0.0, S, u, topk=[1, 30, 33])
+    _check_decode(gl, 0, 0.0, None, None, with_phi=False, topk=[1, 256, 2])
+    # anchors longer than the sequence: everything is an anchor
+    cfg2 = _cfg("c1_1b_4k", n_q_heads=4, n_kv_heads=1)
+    inp2 = make_layer_inputs(cfg2, 9, seq_lens=[3, 68, 70], n_steps=1)
+    gl2 = PU.to_gpu(cfg2, inp2, make_phi_params(cfg2, 9))
+    S2, u2 = PU.gpu_build(gl2)
+    _check_build(gl2, S2, u2)
+    _check_decode(gl2, 0, 0.0, S2, u2, topk=[0, 0, 2])
+    _check_decode(gl2, 0, 0.0, None, None, with_phi=False, topk=[0, 0, 1])
+
+
+def test_exact_ties_break_towards_lower_index():
+    cfg = _cfg("c1_1b_4k", n_q_heads=4, n_kv_heads=1, needles_per_head=0)
+    inp = make_layer_inputs(cfg, 10, seq_lens=[1000], n_steps=1)
+    # every mid key identical -> every score ties exactly; then plant blocks of duplicates
+    inp.k[0, 4:936] = inp.k[0, 4].clone()
+    gl = PU.to_gpu(cfg, inp, make_phi_params(cfg, 10))
+    out = PU.gpu_decode(gl, inp.q[0], np.array([37], np.int32), with_phi=False)
+    assert (out["idx"][0, :, :37] == np.arange(4, 41)).all()
+    inp2 = make_layer_inputs(cfg, 11, seq_lens=[3000], n_steps=1)
+    src = inp2.k[0, 100:110].clone()
+    for rep in range(40):                       # 40 copies of 10 distinct rows, spread out
+        inp2.k[0, 200 + rep * 60: 210 + rep * 60] = src
+    gl2 = PU.to_gpu(cfg, inp2, make_phi_params(cfg, 11))
+    for kk in (5, 57, 203, 411):
+        _check_decode(gl2, 0, 0.0, None, None, with_phi=False, topk=[kk])
+
+
+def test_results_are_run_to_run_identical():
+    cfg = CONFIGS["c1_1b_4k"]
+    inp = make_layer_inputs(cfg, 12, seq_lens=[2500], n_steps=1)
+    gl = PU.to_gpu(cfg, inp, make_phi_params(cfg, 12))
+    S, u = PU.gpu_build(gl)
+    S2, u2 = PU.gpu_build(gl)
+    assert torch.equal(S, S2) and torch.equal(u, u2)
+    a = PU.gpu_decode(gl, inp.q[0], inp.topk(0.02), S, u)
+    b = PU.gpu_decode(gl, inp.q[0], inp.topk(0.02), S, u)
+    assert np.array_equal(a["y"], b["y"]) and np.array_equal(a["idx"], b["idx"])
