@@ -1,0 +1,376 @@
+#!/usr/bin/env python3
+"""Benchmark of the Top-K+phi decode step (128K-context, Llama-3.2-3B head geometry).
+
+One "step" is one decode token through all layers of the workload: per layer one
+call of ``tkphi_decode_step`` (score + select, exact branch, subtraction, residual
+estimate, merge) on one stream.  The prefill summary build is timed separately
+and reported under ``build``.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs an
+independent replica of the same workload on its own GPU: the path has no
+exchange step, so there is no data-path collective; timing is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import CONFIGS, make_layer_inputs, make_phi_params  # noqa: E402
+
+L2_BYTES = 126e6
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons every 100 ms while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._nvml = None
+
+    def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nvml = None
+            return
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def _run(self):
+        nv = self._nvml
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- workload
+def algorithmic_bytes(cfg, n_tokens, topk, n_layers):
+    """Bytes the method itself must move per decode step (the score buffer is an
+    implementation artefact and is not counted)."""
+    d, r = cfg.head_dim, cfg.n_feat
+    n_anchor = cfg.n_sink + cfg.n_tail
+    n_mid = n_tokens - n_anchor
+    key_stream = cfg.n_kv_heads * n_mid * d * 2
+    gather = cfg.n_q_heads * (topk + n_anchor) * 4 * d
+    su = cfg.n_kv_heads * (d * r + r) * 4
+    weights = (cfg.n_q_heads + cfg.n_kv_heads) * (r * d + r) * 4
+    per_layer = key_stream + gather + su + weights
+    return {"key_stream": key_stream * n_layers, "total": per_layer * n_layers,
+            "key_stream_per_layer": key_stream}
+
+
+def run_ours(args, rank, world, device):
+    import paper_2604_05438_b200 as T
+    from paper_2604_05438_b200.build import build_library
+    build_library()
+    T.load_library()
+    cfg = CONFIGS[args.config]
+    n_layers = args.layers or cfg.n_layers
+    N = args.seq_len or cfg.seq_len
+    seed = 0
+    torch.cuda.set_device(device)
+    layers, phis, Ss, us = [], [], [], []
+    t_gen = time.time()
+    for l in range(n_layers):
+        inp = make_layer_inputs(cfg, seed, layer=l, device=device, seq_lens=[N] * cfg.batch, n_steps=1)
+        phi = make_phi_params(cfg, seed + l, device=device)
+        kv = T.KVCache(inp.k, inp.v, inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, cfg.n_sink, cfg.n_tail)
+        layers.append((inp, kv))
+        phis.append(T.PhiMaps(phi.w_q, phi.b_q, phi.w_k, phi.b_k, phi.gamma_q, phi.gamma_k))
+    torch.cuda.synchronize()
+    t_gen = time.time() - t_gen
+    topk = layers[0][0].topk(args.budget)
+    tmax = int(topk.max())
+    topk_dev = torch.from_numpy(topk).to(device)
+    B, Hq, Hkv, d, r = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_feat
+    kv0 = layers[0][1]
+    ws = torch.empty(T.workspace_bytes(kv0, topk, tmax, T.WS_DECODE_STEP), dtype=torch.uint8, device=device)
+    wsb = torch.empty(T.workspace_bytes(kv0, None, 0, T.WS_BUILD), dtype=torch.uint8, device=device)
+
+    # ---- prefill summary build (timed separately)
+    for l in range(n_layers):
+        Ss.append(torch.empty(B, Hkv, d, r, device=device))
+        us.append(torch.empty(B, Hkv, r, device=device))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    T.build_summaries(layers[0][1], phis[0], Ss[0], us[0], wsb)      # warm-up
+    torch.cuda.synchronize()
+    e0.record()
+    for l in range(n_layers):
+        T.build_summaries(layers[l][1], phis[l], Ss[l], us[l], wsb)
+    e1.record()
+    torch.cuda.synchronize()
+    build_ms = e0.elapsed_time(e1)
+
+    # ---- decode queries: a fresh query per step, resident in HBM for the device-timed loop
+    n_q_sets = 8
+    g = torch.Generator(device=device)
+    g.manual_seed(1234)
+    topic_q = [layers[l][0].q[0] for l in range(n_layers)]          # [B,Hq,d] bf16 correlated with needles
+    q_dev = []
+    for s in range(n_q_sets):
+        qs = torch.stack([(topic_q[l].float() + 0.5 * torch.randn(B, Hq, d, generator=g, device=device))
+                          .to(torch.bfloat16) for l in range(n_layers)])
+        q_dev.append(qs.contiguous())                                # [layers,B,Hq,d]
+    y_dev = torch.empty(n_layers, B, Hq, d, device=device)
+
+    def step(qs):
+        for l in range(n_layers):
+            T.decode_step(layers[l][1], phis[l], qs[l], topk, topk_dev, tmax, Ss[l], us[l], None, y_dev[l],
+                          None, 0, ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for w in range(args.warmup):
+        step(q_dev[w % n_q_sets])
+    barrier()
+    sampler = ClockSampler(device.index or 0)
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    ev[0].record()
+    for s in range(args.steps):
+        step(q_dev[s % n_q_sets])
+        ev[s + 1].record()
+    barrier()
+    clocks = sampler.stop()
+    per_step = [ev[s].elapsed_time(ev[s + 1]) for s in range(args.steps)]
+    total_ms = ev[0].elapsed_time(ev[args.steps])
+    assert T.device_status(ws) == 0, "a device-side wait timed out"
+    assert torch.isfinite(y_dev).all()
+
+    # ---- per-kernel durations (second pass with the library's event hooks), for the roofline
+    kt = None
+    if hasattr(T, "kernel_timing"):
+        kt = T.kernel_timing(lambda: [step(q_dev[s % n_q_sets]) for s in range(min(args.steps, 8))])
+
+    # ---- end to end: host buffers, H2D of the queries and D2H of the outputs inside the timed region
+    q_host = [qs.cpu().pin_memory() for qs in q_dev]
+    y_host = torch.empty(n_layers, B, Hq, d).pin_memory()
+    q_stage = torch.empty_like(q_dev[0])
+
+    def step_e2e(s):
+        q_stage.copy_(q_host[s % n_q_sets], non_blocking=True)
+        step(q_stage)
+        y_host.copy_(y_dev, non_blocking=True)
+        torch.cuda.current_stream().synchronize()     # the caller reads y before the next token
+
+    for w in range(min(args.warmup, 3)):
+        step_e2e(w)
+    barrier()
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        step_e2e(s)
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+
+    ms = total_ms / args.steps
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+
+    ab = algorithmic_bytes(cfg, N, tmax, n_layers)
+    peak, peak_kind = _peaks()
+    out = {
+        "metric": "Top-K+phi decode-step latency (us), 128K ctx",
+        "value": ms * 1e3, "unit": "us/step", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 K/V, f32 accumulate", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: {n_layers} layers x {Hq}q/{Hkv}kv heads, d={d}, r={r}, N={N}, "
+                               f"anchors {cfg.n_sink}+{cfg.n_tail}, budget {args.budget:g} (K={tmax}), batch {B}",
+                   "l2": "inputs (K/V of all layers) exceed L2 by >100x; no flush needed",
+                   "replicas": world, "seed": seed},
+        "step_us": {"median": statistics.median(per_step) * 1e3, "min": min(per_step) * 1e3,
+                    "max": max(per_step) * 1e3},
+        "achieved_gbs": ab["total"] / (ms * 1e-3) / 1e9,
+        "hbm_frac_of_measured_peak": ab["total"] / (ms * 1e-3) / 1e9 / peak,
+        "algorithmic_bytes_per_step": ab["total"],
+        "steps_per_s_all_gpus": world * 1e3 / ms,
+        "gpu_launches": args.steps * n_layers * 4,
+        "e2e": {"value": e2e_ms * 1e3, "unit": "us/step", "h2d_bytes_per_step": q_stage.numel() * 2,
+                "d2h_bytes_per_step": y_host.numel() * 4},
+        "build": {"ms_all_layers": build_ms, "kv_bytes": 2 * n_layers * Hkv * (N - cfg.n_sink - cfg.n_tail) * d * 2 * B},
+        "clocks": clocks,
+        "gen_s": t_gen,
+    }
+    if kt is not None:
+        dom = kt["score_hist"]
+        a = ab["key_stream_per_layer"] / (dom["avg_ms"] * 1e-3) / 1e9
+        out["roofline"] = {"bound": "hbm", "kernel": "score_hist_kernel", "achieved": a, "peak": peak,
+                           "unit": "GB/s", "frac": a / peak, "traffic": None, "peak_kind": peak_kind,
+                           "avg_launch_us": dom["avg_ms"] * 1e3}
+        out["kernels_us_per_launch"] = {k: v["avg_ms"] * 1e3 for k, v in kt.items()}
+    return out, (cfg, layers, phis, Ss, us, topk)
+
+
+# --------------------------------------------------------------------------- oracle legs
+def oracle_step_sample(cfg, N, budget, n_heads, seed=0):
+    """Times the float64 oracle (as it stands) on `n_heads` query heads of one layer and
+    scales to a full decode step.  Returns (us_per_step_estimate, seconds_spent, threads)."""
+    from oracle import tkphi_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = 1
+    inp = make_layer_inputs(cfg, seed, layer=0, seq_lens=[N] * cfg.batch, n_steps=1)
+    phi = make_phi_params(cfg, seed)
+    topk = int(inp.topk(budget)[0])
+    G = cfg.group
+    # summaries are prefill state: built outside the timed decode sample
+    built = {}
+    heads = list(range(0, cfg.n_q_heads, max(1, cfg.n_q_heads // n_heads)))[:n_heads]
+    for hq in heads:
+        kvh = hq // G
+        if kvh not in built:
+            K = inp.k[kvh].double().numpy()
+            V = inp.v[kvh].double().numpy()
+            built[kvh] = (K, V) + O.build_summaries(K, V, phi.w_k[kvh].double().numpy(),
+                                                    phi.b_k[kvh].double().numpy(), phi.gamma_k,
+                                                    cfg.n_sink, cfg.n_tail)
+    t0 = time.perf_counter()
+    for hq in heads:
+        kvh = hq // G
+        K, V, S, u = built[kvh]
+        O.topkphi_attention(inp.q[0, 0, hq].double().numpy(), K, V, cfg.n_sink, cfg.n_tail, topk,
+                            phi.w_q[hq].double().numpy(), phi.b_q[hq].double().numpy(), phi.gamma_q,
+                            phi.w_k[kvh].double().numpy(), phi.b_k[kvh].double().numpy(), phi.gamma_k,
+                            S=S, u=u)
+    dt = time.perf_counter() - t0
+    return dt / len(heads) * cfg.n_q_heads * cfg.batch, dt, threads, len(heads)
+
+
+def run_reference(args):
+    cfg = CONFIGS[args.config]
+    n_layers = args.layers or cfg.n_layers
+    N = args.seq_len or cfg.seq_len
+    n_heads = 2
+    vals = []
+    threads = 1
+    for s in range(args.warmup + args.steps):
+        per_layer_s, dt, threads, nh = oracle_step_sample(cfg, N, args.budget, n_heads, seed=s)
+        if s >= args.warmup:
+            vals.append(per_layer_s * n_layers)
+    us = statistics.mean(vals) * 1e6
+    tmax = int(math.floor(args.budget * (N - cfg.n_sink - cfg.n_tail) + 1e-9))
+    sample = (f"{n_heads} of {cfg.n_q_heads} query heads of one layer per step, full N={N}, "
+              f"scaled by heads and {n_layers} layers")
+    return {
+        "impl": "reference", "metric": "Top-K+phi decode-step latency (us), 128K ctx", "value": us,
+        "unit": "us/step", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: {n_layers} layers x {cfg.n_q_heads}q/{cfg.n_kv_heads}kv heads, "
+                               f"d={cfg.head_dim}, r={cfg.n_feat}, N={N}, anchors {cfg.n_sink}+{cfg.n_tail}, "
+                               f"budget {args.budget:g} (K={tmax}), batch {cfg.batch}"},
+        "cpu_baseline": {"value": us, "unit": "us/step", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=32)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c3_3b_128k", choices=sorted(CONFIGS))
+    ap.add_argument("--budget", type=float, default=0.01)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
+    ap.add_argument("--seq-len", type=int, default=0, help="override the context length (profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    device = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=device)
+    out, _ = run_ours(args, rank, world, device)
+    if rank == 0:
+        if not args.no_cpu_baseline:
+            cfg = CONFIGS[args.config]
+            n_layers = args.layers or cfg.n_layers
+            N = args.seq_len or cfg.seq_len
+            per_layer_s, dt, threads, nh = oracle_step_sample(cfg, N, args.budget, 8)
+            out["cpu_baseline"] = {
+                "value": per_layer_s * n_layers * 1e6, "unit": "us/step", "cores": threads, "kind": "oracle",
+                "sample": f"{nh} of {cfg.n_q_heads} query heads of one layer at full N={N} ({dt:.1f} s of oracle "
+                          f"time), scaled by heads and {n_layers} layers; summaries prebuilt"}
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -165,6 +165,26 @@ tkphi_status tkphi_decode_step(const tkphi_kv_desc* kv, const tkphi_phi_desc* ph
  */
 tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32_t* status_out);
 
+/*
+ * Optional per-kernel timing for benchmarks (no counterpart in the paper).  While
+ * enabled, every launch the library makes is bracketed by CUDA events on the caller's
+ * stream (the events are host objects; no device memory is allocated).  Not
+ * thread-safe; leave it off in production.  tkphi_kernel_timing_read waits for the
+ * recorded events, adds up milliseconds and launch counts per kernel kind into the
+ * two host arrays of TKPHI_KERNEL_KINDS entries, and clears the record.
+ */
+enum {
+  TKPHI_KERNEL_SCORE_HIST = 0,      /* key scoring + histogram (streams the mid-region keys) */
+  TKPHI_KERNEL_PARTITION = 1,       /* score bitmaps against the threshold bin */
+  TKPHI_KERNEL_FINALIZE_SELECT = 2, /* exact threshold, ties, ascending index list */
+  TKPHI_KERNEL_EXACT_RESIDUAL = 3,  /* exact branch, subtraction, residual, merge */
+  TKPHI_KERNEL_BUILD = 4,           /* prefill summary build */
+  TKPHI_KERNEL_MEMSET = 5,          /* clearing counters and histograms */
+  TKPHI_KERNEL_KINDS = 6
+};
+void tkphi_kernel_timing_enable(int32_t on);
+tkphi_status tkphi_kernel_timing_read(float* ms_out, int32_t* count_out);
+
 /* Message for the last error returned on the calling thread ("" if none). */
 const char* tkphi_last_error(void);
 

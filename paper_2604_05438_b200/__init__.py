@@ -16,6 +16,8 @@ from .binding import (  # noqa: F401
     topk_decode,
     decode_step,
     device_status,
+    kernel_timing,
+    KERNEL_KINDS,
     WS_BUILD,
     WS_TOPK_DECODE,
     WS_DECODE_STEP,

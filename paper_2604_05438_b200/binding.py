@@ -19,7 +19,9 @@ FLAG_NONE, FLAG_NOSUB = 0, 1
 EXPORTED_SYMBOLS = (
     "tkphi_workspace_bytes", "tkphi_build_summaries", "tkphi_topk_decode", "tkphi_decode_step",
     "tkphi_device_status", "tkphi_last_error", "tkphi_version",
+    "tkphi_kernel_timing_enable", "tkphi_kernel_timing_read",
 )
+KERNEL_KINDS = ("score_hist", "partition", "finalize_select", "exact_residual", "build", "memset")
 
 
 class TkphiError(RuntimeError):
@@ -68,6 +70,10 @@ def load_library():
                                       C.c_void_p, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.tkphi_device_status.restype = C.c_int
     lib.tkphi_device_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+    lib.tkphi_kernel_timing_enable.restype = None
+    lib.tkphi_kernel_timing_enable.argtypes = [C.c_int32]
+    lib.tkphi_kernel_timing_read.restype = C.c_int
+    lib.tkphi_kernel_timing_read.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.tkphi_last_error.restype = C.c_char_p
     lib.tkphi_version.restype = C.c_int32
     _lib = lib
@@ -193,3 +199,20 @@ def device_status(workspace: torch.Tensor, stream=None) -> int:
     out = C.c_int32(0)
     _check(lib.tkphi_device_status(workspace.data_ptr(), _stream_ptr(stream), C.byref(out)))
     return int(out.value)
+
+
+def kernel_timing(fn) -> dict:
+    """Run ``fn()`` with the library's per-kernel event timing on; returns
+    {kind: {"ms": total, "launches": n, "avg_ms": ms/n}} for the kinds that ran."""
+    lib = load_library()
+    lib.tkphi_kernel_timing_enable(1)
+    try:
+        fn()
+        torch.cuda.synchronize()
+        ms = (C.c_float * len(KERNEL_KINDS))()
+        cnt = (C.c_int32 * len(KERNEL_KINDS))()
+        _check(lib.tkphi_kernel_timing_read(ms, cnt))
+    finally:
+        lib.tkphi_kernel_timing_enable(0)
+    return {k: {"ms": float(ms[i]), "launches": int(cnt[i]), "avg_ms": float(ms[i]) / cnt[i]}
+            for i, k in enumerate(KERNEL_KINDS) if cnt[i] > 0}

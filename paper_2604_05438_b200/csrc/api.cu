@@ -6,6 +6,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <vector>
 
 using namespace tkphi;
 
@@ -161,23 +162,43 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 3-D view [head][row][dim] of the key cache; box = one scoring tile of one head.
+// 3-D view [head][row][dim] of the key cache; box = 64 dims x one scoring tile of one
+// head, stored with the 128-byte swizzle (head_dim 128 takes two boxes per tile).
 tkphi_status make_key_tensor_map(const tkphi_kv_desc* kv, long long total_tokens, CUtensorMap* tm) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return fail(TKPHI_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   const cuuint64_t dims[3] = {(cuuint64_t)kv->head_dim, (cuuint64_t)total_tokens, (cuuint64_t)kv->n_kv_heads};
   const cuuint64_t strides[2] = {(cuuint64_t)kv->kv_stride_token * 2, (cuuint64_t)kv->kv_stride_head * 2};
-  const cuuint32_t box[3] = {(cuuint32_t)kv->head_dim, (cuuint32_t)score_tile_keys(kv->head_dim), 1};
+  const cuuint32_t box[3] = {64, (cuuint32_t)score_tile_keys(kv->head_dim), 1};   // 128-byte rows
   const cuuint32_t estr[3] = {1, 1, 1};
   // a single head (stride 0 would be rejected): give the unused dimension a legal stride
   cuuint64_t st[2] = {strides[0], strides[1]};
   if (kv->n_kv_heads == 1 || st[1] == 0) st[1] = st[0] * (cuuint64_t)total_tokens;
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(kv->k), dims, st, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(TKPHI_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
   return TKPHI_OK;
 }
+
+// ---- optional per-kernel timing (off by default): CUDA events around every launch
+struct TimedSpan { cudaEvent_t a, b; int kind; };
+bool g_timing = false;
+std::vector<TimedSpan> g_spans;
+
+struct ScopedSpan {
+  cudaStream_t st; int kind; cudaEvent_t a = nullptr, b = nullptr;
+  ScopedSpan(cudaStream_t s, int k) : st(s), kind(k) {
+    if (!g_timing) return;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { a = b = nullptr; return; }
+    cudaEventRecord(a, st);
+  }
+  ~ScopedSpan() {
+    if (!a) return;
+    cudaEventRecord(b, st);
+    g_spans.push_back({a, b, kind});
+  }
+};
 
 tkphi_status check_ws(void* ws, size_t have, size_t need) {
   if (!ws) return fail(TKPHI_ERR_WORKSPACE, "workspace is NULL");
@@ -248,7 +269,11 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   // idx_out uses the caller's topk_max as its row length; the internal list uses p.topk_max
   if (topk_max == 0) p.idx_out = nullptr;
 
-  cudaError_t e = cudaMemsetAsync(w, 0, L.zero_end, cs);
+  cudaError_t e;
+  {
+    ScopedSpan sp(cs, TKPHI_KERNEL_MEMSET);
+    e = cudaMemsetAsync(w, 0, L.zero_end, cs);
+  }
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
   if (sh.score_tiles > 0) {
     CUtensorMap tm;
@@ -256,15 +281,25 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
     if (st != TKPHI_OK) return st;
     long long grid = sh.score_tiles < n_sm_cached() ? sh.score_tiles : n_sm_cached();
     for (int pass = 0; pass < L.passes; ++pass) {
+      ScopedSpan sp(cs, TKPHI_KERNEL_SCORE_HIST);
       e = launch_score_hist(p, tm, pass, (int)grid, cs);
       if (e != cudaSuccess) return cuda_fail(e, "score_hist launch");
     }
-    e = launch_partition(p, sh.max_mid, cs);
+    {
+      ScopedSpan sp(cs, TKPHI_KERNEL_PARTITION);
+      e = launch_partition(p, sh.max_mid, cs);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "partition launch");
   }
-  e = launch_finalize_select(p, cs);
+  {
+    ScopedSpan sp(cs, TKPHI_KERNEL_FINALIZE_SELECT);
+    e = launch_finalize_select(p, cs);
+  }
   if (e != cudaSuccess) return cuda_fail(e, "finalize_select launch");
-  e = launch_exact_residual(p, cs);
+  {
+    ScopedSpan sp(cs, TKPHI_KERNEL_EXACT_RESIDUAL);
+    e = launch_exact_residual(p, cs);
+  }
   if (e != cudaSuccess) return cuda_fail(e, "exact_residual launch");
   return TKPHI_OK;
 }
@@ -323,7 +358,10 @@ tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc
   p.chunk_len = L.chunk_len; p.chunks_per_unit = L.chunks_per_unit;
   cudaError_t e = cudaMemsetAsync(w, 0, L.zero_end, cs);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
-  e = launch_build(p, cs);
+  {
+    ScopedSpan sp(cs, TKPHI_KERNEL_BUILD);
+    e = launch_build(p, cs);
+  }
   if (e != cudaSuccess) return cuda_fail(e, "build launch");
   return TKPHI_OK;
 }
@@ -351,6 +389,32 @@ tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32
   if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
   if (e != cudaSuccess) return cuda_fail(e, "reading the device status word");
   return TKPHI_OK;
+}
+
+void tkphi_kernel_timing_enable(int32_t on) {
+  g_timing = on != 0;
+  if (!g_timing) {
+    for (auto& sp : g_spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    g_spans.clear();
+  }
+}
+
+tkphi_status tkphi_kernel_timing_read(float* ms_out, int32_t* count_out) {
+  g_err[0] = 0;
+  if (!ms_out || !count_out) return fail(TKPHI_ERR_INVALID_ARG, "NULL argument");
+  for (int i = 0; i < TKPHI_KERNEL_KINDS; ++i) { ms_out[i] = 0.f; count_out[i] = 0; }
+  tkphi_status st = TKPHI_OK;
+  for (auto& sp : g_spans) {
+    float ms = 0.f;
+    cudaError_t e = cudaEventSynchronize(sp.b);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, sp.a, sp.b);
+    if (e != cudaSuccess) st = cuda_fail(e, "reading a timing event");
+    else { ms_out[sp.kind] += ms; count_out[sp.kind] += 1; }
+    cudaEventDestroy(sp.a);
+    cudaEventDestroy(sp.b);
+  }
+  g_spans.clear();
+  return st;
 }
 
 }  // extern "C"

@@ -4,8 +4,8 @@
 // broken towards the lower index (exhaustive Top-K control selector, Sec. 5.1).
 //
 // Three kernels:
-//   score_hist_kernel      streams the keys once (TMA-staged tiles, 4-stage mbarrier
-//                          ring), writes fp32 scores and a 4096-bin histogram of the
+//   score_hist_kernel      streams the keys once (TMA-staged 128B-swizzled tiles, 4-stage
+//                          mbarrier ring), writes fp32 scores and a 4096-bin histogram of the
 //                          leading 12 bits of the order-preserving score key; the last
 //                          CTA to finish a (sequence, KV head) unit turns the histogram
 //                          into a threshold bin per query head.
@@ -165,19 +165,26 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
     for (; issued < kScoreStages && f0 + issued < f1; ++issued) {
       mbar_expect_tx(&full[issued], kScoreTileBytes);
       int row = (int)(p.cu_seqlens[pc.b] + p.n_sink) + pc.t * TK;
-      tma_load_3d(tiles + issued * kScoreTileBytes, &tmap_k, &full[issued], 0, row, pc.kvh);
+#pragma unroll
+      for (int x = 0; x < D / 64; ++x)
+        tma_load_3d(tiles + issued * kScoreTileBytes + x * (TK * 128), &tmap_k, &full[issued], x * 64, row, pc.kvh);
       cursor_next(pc, pre, batch, n_kv);
     }
   }
 
-  // ---- per-thread geometry: key slice and bank-conflict-free chunk rotation
-  const int s = tid % LPK;                  // 32-dim slice of the key handled by this lane
-  const int kk = tid / LPK;                 // key within a pass
-  const int rho = (LPK == 2) ? ((lane >> 1) & 3) : (((s >> 1) + 2 * ((lane >> 2) & 1)) & 3);
+  // ---- per-thread geometry.  Tiles are stored with the 128-byte TMA swizzle: the
+  // 16-byte chunk c of row r sits at chunk position c ^ (r & 7).  The eight lanes
+  // of a shared-memory access phase read the same logical chunk of eight
+  // consecutive rows, so they hit eight different positions: no bank conflicts,
+  // and every key is accumulated in the same (natural) order wherever it sits.
+  constexpr int KPW = 32 / LPK;             // keys per warp and pass
+  const int s = lane / KPW;                 // 32-dim slice of the key handled by this lane
+  const int kk = (tid >> 5) * KPW + (lane % KPW);   // key within a pass
+  const int sub_off = (s >> 1) * (TK * 128);        // D = 128: second 64-dim half is a second box
   int coff[4];
 #pragma unroll
-  for (int c = 0; c < 4; ++c) coff[c] = s * 64 + (((c + rho) & 3) << 4);
-  const int offA = kk * (2 * D), offB = (kk + KPP) * (2 * D);
+  for (int c = 0; c < 4; ++c) coff[c] = ((((s & 1) * 4 + c) ^ (kk & 7)) << 4);
+  const int offA = sub_off + kk * 128, offB = sub_off + (kk + KPP) * 128;   // KPP % 8 == 0
 
   TileCursor cc;
   cursor_seek(cc, pre, batch, n_kv, f0);
@@ -241,13 +248,13 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
       len_b = p.cu_seqlens[cur_b + 1] - cu_b;
       n_mid = mid_len(len_b, p.n_sink, p.n_tail);
       row_base0 = score_row_base(p, cur_b, cur_kvh * p.group + g0, cu_b, len_b);
-      // this lane's slice of the G queries, in the same rotated chunk order as the key loads
+      // this lane's 32-dim slice of the G queries
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         const __nv_bfloat16* qp = p.q + ((size_t)cur_b * p.n_q_heads + cur_kvh * p.group + g0 + g) * D + s * 32;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const uint4 raw = *reinterpret_cast<const uint4*>(qp + (((c + rho) & 3) << 3));
+          const uint4 raw = *reinterpret_cast<const uint4*>(qp + (c << 3));
           const unsigned w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
@@ -287,7 +294,7 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
 #pragma unroll
     for (int g = 0; g < G; ++g) {
 #pragma unroll
-      for (int o = 1; o < LPK; o <<= 1) {
+      for (int o = KPW; o < 32; o <<= 1) {
         acc[0][g] += __shfl_xor_sync(0xffffffffu, acc[0][g], o);
         acc[1][g] += __shfl_xor_sync(0xffffffffu, acc[1][g], o);
       }
@@ -325,7 +332,9 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
     if (tid == 0 && f0 + issued < f1) {
       mbar_expect_tx(&full[slot], kScoreTileBytes);
       int row = (int)(p.cu_seqlens[pc.b] + p.n_sink) + pc.t * TK;
-      tma_load_3d(tiles + slot * kScoreTileBytes, &tmap_k, &full[slot], 0, row, pc.kvh);
+#pragma unroll
+      for (int x = 0; x < D / 64; ++x)
+        tma_load_3d(tiles + slot * kScoreTileBytes + x * (TK * 128), &tmap_k, &full[slot], x * 64, row, pc.kvh);
       cursor_next(pc, pre, batch, n_kv);
       ++issued;
     }

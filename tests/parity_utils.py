@@ -18,6 +18,7 @@ SU_TOL = 1e-3         # max |S_hat - S| / max |S| per head (same for u)
 TIE_TOL = 1e-5        # index sets may differ only where |s_i - tau| <= TIE_TOL * max(|tau|, 1)
 LOGZ_TOL = 2e-3       # absolute, on log Z_hat_R
 ME_TOL = 1e-4         # absolute, on the exact-branch max score
+FP32_TINY = 1.2e-38   # below the smallest normal fp32 a summary entry is not representable
 
 
 def max_rel(a, b) -> float:
