@@ -119,6 +119,36 @@ tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Prefill summary build without any caller-provided workspace (the paper has no
+ * counterpart; this serves a deployment constraint).  Some callers cannot obtain
+ * device memory at call time: plug-ins of a serving process whose memory pool is sized
+ * and handed out once at start-up, runtimes that forbid cudaMalloc (an implicit
+ * device-wide synchronisation) on the latency-critical path, and hosts whose policy
+ * allows allocation only during initialisation.  For them this entry point
+ * computes exactly what tkphi_build_summaries computes, on the same kernel, but takes
+ * its scratch from a fixed array of TKPHI_STATIC_SCRATCH_BYTES that is part of the
+ * library's device image.  It calls no allocating routine of CUDA or of any library.
+ *  - Limit: problems whose tkphi_workspace_bytes(kv, NULL, 0, TKPHI_WS_BUILD) exceeds
+ *    TKPHI_STATIC_SCRATCH_BYTES are rejected with TKPHI_ERR_WORKSPACE before anything
+ *    is enqueued (the message names both sizes); use tkphi_build_summaries for those.
+ *  - Cost: every GPU on which the library is loaded holds the array until the process
+ *    exits, whether or not this function is ever called.
+ *  - First call on each device: looks up the array's device address (a host-side
+ *    runtime query, done with that device current and cached).  Make that first call
+ *    before any stream capture begins on the device.
+ *  - Sharing: all calls on a device use the same array.  The array keeps the previous
+ *    call's contents; the part that must start at zero is cleared on the stream at the
+ *    start of every call.  Two calls whose GPU work overlaps (different streams, or
+ *    different host threads) race on it and give undefined results: serialise them.
+ * Arguments, outputs and error reporting otherwise as for tkphi_build_summaries;
+ * tkphi_static_last_error() gives the message of the last failing call of the thread.
+ */
+#define TKPHI_STATIC_SCRATCH_BYTES (8u << 20)
+tkphi_status tkphi_build_summaries_static(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi,
+                                          float* S, float* u, void* cuda_stream);
+const char* tkphi_static_last_error(void);
+
+/*
  * Selection-only Top-K decode (Sec. 3, Eq. exact_terms and y_TopK = nu_E / Z_E), steps
  * (1)-(2) above.
  *   q         bf16 [batch][n_q_heads][head_dim], one decode query per sequence and head.

@@ -13,6 +13,8 @@ from .binding import (  # noqa: F401
     library_path,
     workspace_bytes,
     build_summaries,
+    build_summaries_static,
+    STATIC_SCRATCH_BYTES,
     topk_decode,
     decode_step,
     device_status,

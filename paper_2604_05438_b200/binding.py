@@ -20,7 +20,9 @@ EXPORTED_SYMBOLS = (
     "tkphi_workspace_bytes", "tkphi_build_summaries", "tkphi_topk_decode", "tkphi_decode_step",
     "tkphi_device_status", "tkphi_last_error", "tkphi_version",
     "tkphi_kernel_timing_enable", "tkphi_kernel_timing_read",
+    "tkphi_build_summaries_static", "tkphi_static_last_error",
 )
+STATIC_SCRATCH_BYTES = 8 << 20
 KERNEL_KINDS = ("score_hist", "partition", "finalize_select", "exact_residual", "build", "memset")
 
 
@@ -61,6 +63,10 @@ def load_library():
     lib.tkphi_build_summaries.restype = C.c_int
     lib.tkphi_build_summaries.argtypes = [C.POINTER(_KvDesc), C.POINTER(_PhiDesc), C.c_void_p, C.c_void_p,
                                           C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.tkphi_build_summaries_static.restype = C.c_int
+    lib.tkphi_build_summaries_static.argtypes = [C.POINTER(_KvDesc), C.POINTER(_PhiDesc), C.c_void_p, C.c_void_p,
+                                                 C.c_void_p]
+    lib.tkphi_static_last_error.restype = C.c_char_p
     lib.tkphi_topk_decode.restype = C.c_int
     lib.tkphi_topk_decode.argtypes = [C.POINTER(_KvDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -168,6 +174,17 @@ def build_summaries(kv: KVCache, phi: PhiMaps, S: torch.Tensor, u: torch.Tensor,
     _check(lib.tkphi_build_summaries(C.byref(d), C.byref(ph), S.data_ptr(), u.data_ptr(),
                                      workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                      _stream_ptr(stream)))
+
+
+def build_summaries_static(kv: KVCache, phi: PhiMaps, S: torch.Tensor, u: torch.Tensor, stream=None) -> None:
+    """Summary build on the library's built-in scratch: for callers that may not
+    allocate device memory.  Problems needing more than STATIC_SCRATCH_BYTES of
+    scratch raise TkphiError (status -3).  Calls that overlap on the GPU race."""
+    lib = load_library()
+    d, ph = kv.desc(), phi.desc()
+    st = lib.tkphi_build_summaries_static(C.byref(d), C.byref(ph), S.data_ptr(), u.data_ptr(), _stream_ptr(stream))
+    if st != 0:
+        raise TkphiError(st, lib.tkphi_static_last_error().decode())
 
 
 def topk_decode(kv: KVCache, q: torch.Tensor, topk_host, topk_dev: torch.Tensor, topk_max: int,

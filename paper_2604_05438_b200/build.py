@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtkphi.so")
-SOURCES = ["api.cu", "score_select.cu", "exact_residual.cu", "build_summaries.cu"]
+SOURCES = ["api.cu", "score_select.cu", "exact_residual.cu", "build_summaries.cu", "static_scratch.cu"]
 HEADERS = ["common.cuh", os.path.join("..", "..", "include", "tkphi.h")]
 
 
