@@ -205,7 +205,7 @@ tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32
  */
 enum {
   TKPHI_KERNEL_SCORE_HIST = 0,      /* key scoring + histogram (streams the mid-region keys) */
-  TKPHI_KERNEL_PARTITION = 1,       /* score bitmaps against the threshold bin */
+  TKPHI_KERNEL_COMPACT = 1,         /* bitmap and candidate lists against the threshold bin; phi_q; W_k split */
   TKPHI_KERNEL_FINALIZE_SELECT = 2, /* exact threshold, ties, ascending index list */
   TKPHI_KERNEL_EXACT_RESIDUAL = 3,  /* exact branch, subtraction, residual, merge */
   TKPHI_KERNEL_BUILD = 4,           /* prefill summary build */

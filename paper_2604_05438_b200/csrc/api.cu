@@ -88,6 +88,9 @@ tkphi_status validate_topk(const tkphi_kv_desc* kv, const int32_t* topk_host, in
     if (!allow_empty_support && topk_host[b] == 0 && kv->n_sink == 0 && kv->n_tail == 0)
       return fail(TKPHI_ERR_INVALID_ARG, "sequence %d has an empty exact support (no anchors, topk = 0)", b);
     if (topk_host[b] > 0) sh->score_tiles += (int64_t)kv->n_kv_heads * ((mid + tk - 1) / tk);
+    if (mid > (int64_t)kMaxChunks * kCompactChunk)
+      return fail(TKPHI_ERR_UNSUPPORTED, "sequence %d: mid-region of %lld tokens exceeds %lld", b, (long long)mid,
+                  (long long)kMaxChunks * kCompactChunk);
   }
   if (sh->score_tiles >= (1ll << 31)) return fail(TKPHI_ERR_UNSUPPORTED, "too many key tiles");
   return TKPHI_OK;
@@ -116,7 +119,10 @@ void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, W
   L->scores = o;        o = align_up(o + sizeof(float) * (size_t)kv->n_q_heads * sh.total_tokens, 256);
   const size_t bm_words = ((size_t)kv->n_q_heads * sh.total_tokens) / 32 + sh.rows + 2;
   L->bm_sure = o;       o = align_up(o + 4 * bm_words, 256);
-  L->bm_cand = o;       o = align_up(o + 4 * bm_words, 256);
+  L->cand = o;          o = align_up(o + sizeof(int) * (size_t)kv->n_q_heads * sh.total_tokens, 256);
+  L->max_chunks = sh.max_mid > 0 ? (sh.max_mid + kCompactChunk - 1) / kCompactChunk : 1;
+  L->chunk_ncand = o;   o = align_up(o + sizeof(int) * (size_t)sh.rows * L->max_chunks, 256);
+  L->wk_img = o;        o = align_up(o + (size_t)kv->n_kv_heads * 2 * kv->n_feat * kv->head_dim * 2, 1024);
   L->idx = o;           o = align_up(o + sizeof(int) * (size_t)sh.rows * (topk_max > 0 ? topk_max : 1), 256);
   L->aq = o;            o = align_up(o + sizeof(float) * (size_t)sh.rows * (kv->n_feat + 4), 256);
   int64_t max_support = (int64_t)kv->n_sink + kv->n_tail + topk_max;
@@ -260,7 +266,10 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   p.hist = reinterpret_cast<unsigned*>(w + L.hist);
   p.scores = reinterpret_cast<float*>(w + L.scores);
   p.bm_sure = reinterpret_cast<unsigned*>(w + L.bm_sure);
-  p.bm_cand = reinterpret_cast<unsigned*>(w + L.bm_cand);
+  p.cand = reinterpret_cast<int*>(w + L.cand);
+  p.chunk_ncand = reinterpret_cast<int*>(w + L.chunk_ncand);
+  p.max_chunks = L.max_chunks;
+  p.wk_img = reinterpret_cast<__nv_bfloat16*>(w + L.wk_img);
   p.idx = reinterpret_cast<int*>(w + L.idx);
   p.aq = reinterpret_cast<float*>(w + L.aq);
   p.partials = reinterpret_cast<float*>(w + L.partials);
@@ -285,12 +294,12 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
       e = launch_score_hist(p, tm, pass, (int)grid, cs);
       if (e != cudaSuccess) return cuda_fail(e, "score_hist launch");
     }
-    {
-      ScopedSpan sp(cs, TKPHI_KERNEL_PARTITION);
-      e = launch_partition(p, sh.max_mid, cs);
-    }
-    if (e != cudaSuccess) return cuda_fail(e, "partition launch");
   }
+  {
+    ScopedSpan sp(cs, TKPHI_KERNEL_COMPACT);
+    e = launch_compact(p, sh.score_tiles > 0 ? sh.max_mid : 0, cs);
+  }
+  if (e != cudaSuccess) return cuda_fail(e, "compact launch");
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_FINALIZE_SELECT);
     e = launch_finalize_select(p, cs);

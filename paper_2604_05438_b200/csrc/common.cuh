@@ -14,8 +14,9 @@ constexpr int kHistBits = 12;                 // leading bits of the ordered sco
 constexpr int kHistBins = 1 << kHistBits;     // bins of the fused first-pass histogram
 constexpr int kLowBits = 32 - kHistBits;      // bits refined inside the threshold bin
 constexpr int kMaxBatch = 4096;               // sequences per call
-constexpr int kSlice = 64;                    // exact-support tokens per CTA of the exact/residual kernel
-constexpr uint32_t kSpinLimit = 1u << 22;     // polls of a bounded mbarrier wait (with back-off)
+constexpr int kSlice = 128;                   // exact-support tokens per CTA of the exact/residual kernel (= MMA M)
+constexpr int kCompactChunk = 4096;           // scores per CTA of the compaction kernel
+constexpr int kMaxChunks = 2048;              // compaction chunks per sequence the selection kernel can index
 
 // Device status word values (first word of the workspace).
 constexpr int kStatusOk = 0;
@@ -47,8 +48,11 @@ struct Problem {
   int4* rowinfo;                   // [rows]: x = threshold bin, y = count above, z = count in bin
   unsigned* hist;                  // [rows][kHistBins]
   float* scores;                   // [n_q_heads * total_tokens]
-  unsigned* bm_sure;               // bitmap of surely selected mid positions
-  unsigned* bm_cand;               // bitmap of threshold-bin candidates
+  unsigned* bm_sure;               // bitmap of selected mid positions (first: those above the threshold bin)
+  int* cand;                       // threshold-bin candidates (mid offsets), one segment per compaction chunk
+  int* chunk_ncand;                // [rows][max_chunks] candidates per chunk
+  int max_chunks;
+  __nv_bfloat16* wk_img;           // [n_kv_heads][2][r*d] W_k split into bf16 hi / lo, stored as MMA operand tiles
   int* idx;                        // [rows][topk_max] ascending retrieved positions
   float* aq;                       // [rows][n_feat + 4]: exp(a_q - m_q) per feature, then m_q
   float* partials;                 // [rows][max_slices][partial_stride]
@@ -74,8 +78,8 @@ struct BuildProblem {
 // Host-side byte offsets of the workspace pieces.
 struct WsLayout {
   size_t status, unit_counter, row_counter, hist, zero_end;
-  size_t rowinfo, scores, bm_sure, bm_cand, idx, aq, partials, total;
-  int max_slices, partial_stride, passes;
+  size_t rowinfo, scores, bm_sure, cand, chunk_ncand, wk_img, idx, aq, partials, total;
+  int max_slices, partial_stride, passes, max_chunks;
   // build
   size_t b_partials; int chunk_len, chunks_per_unit;
 };
@@ -159,7 +163,7 @@ __device__ __forceinline__ long long bitmap_row_base(const Problem& p, int b, in
 // ---------------------------------------------------------------- host launchers
 // Each returns cudaGetLastError() after enqueuing on `stream`.
 cudaError_t launch_score_hist(const Problem& p, const CUtensorMap& tmap_k, int pass, int n_sm, cudaStream_t stream);
-cudaError_t launch_partition(const Problem& p, int max_mid, cudaStream_t stream);
+cudaError_t launch_compact(const Problem& p, int max_mid, cudaStream_t stream);
 cudaError_t launch_finalize_select(const Problem& p, cudaStream_t stream);
 cudaError_t launch_exact_residual(const Problem& p, cudaStream_t stream);
 cudaError_t launch_build(const BuildProblem& p, cudaStream_t stream);

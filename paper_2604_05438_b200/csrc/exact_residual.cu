@@ -13,46 +13,58 @@
 // retrieved token contribute to both branches while its v row is in shared memory.
 // phi_q is carried as exp(a_q - m_q) with the log-scale m_q separate.
 //
-// The support list of a query head is cut into slices of kSlice tokens; one CTA
-// per slice writes partial sums, and the last CTA of a head (one atomic ticket, no
-// spinning) combines them in slice order, so results are run-to-run identical.
+// The support list of a query head is cut into slices of 128 tokens, one CTA each.
+// The k and v rows of a slice are gathered into 128B-swizzled shared-memory tiles.
+// The feature recompute of the retrieved keys, W_k k_i for 128 tokens x r features, is
+// a dense [128 x d] x [d x r] contraction: it runs as tcgen05.mma with the gathered key
+// tile as A and W_k, split into bf16 hi + lo parts (two accumulating MMAs, error
+// ~2^-18 |W|), as B; the 128 x r fp32 result stays in tensor memory and each thread
+// reads the row of its own token, so <phi_q, phi_k(k_i)> needs no cross-thread
+// reduction.  Each CTA writes partial sums; the last CTA of a head (one atomic
+// ticket, no spinning) combines them in slice order, so results are run-to-run
+// identical.
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace tkphi {
 
-constexpr int kExThreads = 256;
+constexpr int kExThreads = 128;      // one thread per token of the slice = per tensor-memory lane
 
 template <int D, int R>
 struct ExSmem {
-  static constexpr int WT_LD = R + 1;                       // padded leading dim of W^T
-  static constexpr size_t wt = 0;                           // float [D][R+1]   (phi only)
-  static constexpr size_t kf = wt + sizeof(float) * D * WT_LD;     // float [D][kSlice]
-  static constexpr size_t vs = kf + sizeof(float) * D * kSlice;    // bf16  [kSlice][D]
-  static constexpr size_t red = vs + 2 * kSlice * D;               // float [4][2*D]
-  static constexpr size_t zpart = red + sizeof(float) * 4 * 2 * D; // float [8][kSlice]
-  static constexpr size_t small = zpart + sizeof(float) * 8 * kSlice;
-  // small: tok[kSlice] int, isret[kSlice] int, sc[kSlice], wgt[kSlice], zt[kSlice], knorm[kSlice], qf[D], phiq[R], misc[16]
-  static constexpr size_t total = small + 4 * (6 * kSlice + D + R + 16);
+  static constexpr int BOXES = D / 64;
+  static constexpr int KV_BOX = kSlice * 128;                 // bytes of one 64-dim column block of k or v
+  static constexpr int W_BOX = R * 128;
+  static constexpr size_t kt = 0;                             // bf16 k tile  [BOXES][128][128 B]
+  static constexpr size_t vt = kt + (size_t)BOXES * KV_BOX;   // bf16 v tile
+  static constexpr size_t whi = vt + (size_t)BOXES * KV_BOX;  // bf16 W_k hi  [BOXES][R][128 B]
+  static constexpr size_t wlo = whi + (size_t)BOXES * W_BOX;
+  static constexpr size_t small = wlo + (size_t)BOXES * W_BOX;
+  // small: bars[2] (16 B), tok[128] int, isret[128] int, wgt[128], zt[128], qf[D], phiq[R], bk[R],
+  //        red[4*D], misc[16]
+  static constexpr size_t total = small + 16 + 4 * (4 * kSlice + D + 2 * R + 4 * D + 16);
 };
 
 template <int D, int R>
 __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Problem p) {
   using L = ExSmem<D, R>;
-  extern __shared__ __align__(16) unsigned char smem[];
-  float* Wt = reinterpret_cast<float*>(smem + L::wt);
-  float* kf = reinterpret_cast<float*>(smem + L::kf);
-  __nv_bfloat16* vs = reinterpret_cast<__nv_bfloat16*>(smem + L::vs);
-  float* red = reinterpret_cast<float*>(smem + L::red);
-  float* zpart = reinterpret_cast<float*>(smem + L::zpart);
-  int* tok = reinterpret_cast<int*>(smem + L::small);
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* kt = smem + L::kt;
+  unsigned char* vt = smem + L::vt;
+  unsigned char* whi = smem + L::whi;
+  unsigned char* wlo = smem + L::wlo;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::small);   // [0]: W tiles landed, [1]: MMAs done
+  int* tok = reinterpret_cast<int*>(bars + 2);
   int* isret = tok + kSlice;
-  float* sc = reinterpret_cast<float*>(isret + kSlice);
-  float* wgt = sc + kSlice;
+  float* wgt = reinterpret_cast<float*>(isret + kSlice);
   float* zt = wgt + kSlice;
-  float* knorm = zt + kSlice;
-  float* qf = knorm + kSlice;
+  float* qf = zt + kSlice;
   float* phiq = qf + D;
-  float* misc = phiq + R;
+  float* bk = phiq + R;
+  float* red = bk + R;
+  float* misc = red + 4 * D;
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 12);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 13);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.z, hq = blockIdx.y, slice = blockIdx.x;
@@ -68,13 +80,23 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   const int n_slices = nE > 0 ? (nE + kSlice - 1) / kSlice : 1;
   if (slice >= n_slices) return;
   const bool do_phi = p.with_phi && !(p.flags & 1u);
+  // does this slice hold retrieved tokens (positions nA1 .. nA1+K-1 of the support list)?
+  const bool has_ret = do_phi && slice * kSlice < nA1 + K && (slice + 1) * kSlice > nA1;
 
   const __nv_bfloat16* kbase = p.k + (long long)kvh * p.stride_head + cu_b * p.stride_token;
   const __nv_bfloat16* vbase = p.v + (long long)kvh * p.stride_head + cu_b * p.stride_token;
   const float* srow = p.scores + score_row_base(p, b, hq, cu_b, len_b);
 
+  // ---- 0. barriers, tensor memory, W_k operand tiles
+  if (tid == 0) {
+    mbar_init(&bars[0], 1);
+    mbar_init(&bars[1], 1);
+    mbar_fence_init();
+    *s_abort = 0;
+  }
+  if (has_ret && warp == 0) tmem_alloc(s_tmem, R);
   // ---- 1. token list of this slice
-  if (tid < kSlice) {
+  {
     const int pi = slice * kSlice + tid;
     int t = -1, ret = 0;
     if (pi < nE) {
@@ -87,113 +109,128 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   }
   for (int c = tid; c < D; c += kExThreads) qf[c] = __bfloat162float(p.q[(size_t)row * D + c]);
   if (do_phi) {
-    for (int j = tid; j < R; j += kExThreads) phiq[j] = p.aq[(size_t)row * (R + 4) + j];
-    // W_k^T into shared memory: global reads run along a row of W_k, the padded
-    // leading dimension keeps the transposed stores conflict-free
-    const float* W = p.w_k + (size_t)kvh * R * D;
-    for (int i = tid; i < R * D; i += kExThreads) {
-      const int j = i / D, c = i % D;
-      Wt[c * L::WT_LD + j] = W[i];
+    for (int j = tid; j < R; j += kExThreads) {
+      phiq[j] = p.aq[(size_t)row * (R + 4) + j];
+      bk[j] = p.b_k[(size_t)kvh * R + j];
     }
   }
+  tc_fence_before_sync();
   __syncthreads();
+  tc_fence_after_sync();
+  if (has_ret && tid == 0) {
+    const unsigned char* img = reinterpret_cast<const unsigned char*>(p.wk_img + (size_t)kvh * 2 * R * D);
+    mbar_expect_tx(&bars[0], 2u * R * D * 2u);
+    bulk_load(whi, img, R * D * 2, &bars[0]);
+    bulk_load(wlo, img + (size_t)R * D * 2, R * D * 2, &bars[0]);
+  }
 
-  // ---- 2. gather rows: v always; k for anchors (scores) and, with phi, retrieved rows
+  // ---- 2. gather rows into swizzled tiles: v always; k for anchors (scores) and, with phi,
+  // retrieved rows.  Sixteen-byte asynchronous copies, all in flight at once.
   constexpr int CPR = D / 8;                 // 16-byte chunks per row
   for (int i = tid; i < kSlice * CPR; i += kExThreads) {
     const int t = i / CPR, c = i % CPR;
     const int ti = tok[t];
-    uint4 vraw = make_uint4(0, 0, 0, 0), kraw = make_uint4(0, 0, 0, 0);
+    const uint32_t off = (c >> 3) * L::KV_BOX + swz128(t, c & 7);
     if (ti >= 0) {
-      vraw = *reinterpret_cast<const uint4*>(vbase + (long long)ti * p.stride_token + c * 8);
-      if (!isret[t] || do_phi)
-        kraw = *reinterpret_cast<const uint4*>(kbase + (long long)ti * p.stride_token + c * 8);
-    }
-    *reinterpret_cast<uint4*>(vs + t * D + c * 8) = vraw;
-    const unsigned w[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      kf[(c * 8 + 2 * e) * kSlice + t] = bf16_lo(w[e]);
-      kf[(c * 8 + 2 * e + 1) * kSlice + t] = bf16_hi(w[e]);
+      cp_async_16(vt + off, vbase + (long long)ti * p.stride_token + c * 8);
+      if (!isret[t] || do_phi) cp_async_16(kt + off, kbase + (long long)ti * p.stride_token + c * 8);
+      else *reinterpret_cast<uint4*>(kt + off) = make_uint4(0, 0, 0, 0);
+    } else {
+      *reinterpret_cast<uint4*>(vt + off) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(kt + off) = make_uint4(0, 0, 0, 0);
     }
   }
+  cp_async_wait_all();
+  fence_proxy_async_smem();
   __syncthreads();
 
-  // ---- 3. scores, slice max, softmax weights
-  if (tid < kSlice) {
-    const int ti = tok[tid];
-    float s_val = -INFINITY, kn = 0.f;
-    if (ti >= 0) {
-      float dot = 0.f;
-      for (int c = 0; c < D; ++c) {
-        const float x = kf[c * kSlice + tid];
-        dot = fmaf(x, qf[c], dot);
-        kn = fmaf(x, x, kn);
+  // ---- 3. feature recompute on the tensor core: acc[t][j] = sum_c k_t[c] (W_hi + W_lo)[j][c]
+  bool ok = true;
+  if (has_ret && tid == 0) {
+    ok = mbar_wait(&bars[0], 0, s_abort);
+    if (ok) {
+      tc_fence_after_sync();
+      constexpr uint32_t idesc = umma_idesc_bf16(128, R, 0, 0);
+      const uint32_t tmem_d = *s_tmem;
+      const uint32_t ka = smem_u32(kt);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t wa = smem_u32(half == 0 ? whi : wlo);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint64_t adesc = umma_smem_desc(ka + (k >> 2) * L::KV_BOX + (k & 3) * 32, 16, 1024);
+          const uint64_t bdesc = umma_smem_desc(wa + (k >> 2) * L::W_BOX + (k & 3) * 32, 16, 1024);
+          umma_ss(tmem_d, adesc, bdesc, idesc, (half | k) ? 1u : 0u);
+        }
       }
-      s_val = isret[tid] ? srow[ti - p.n_sink] : dot * p.scale;
+      tc_commit(&bars[1]);
     }
-    sc[tid] = s_val;
-    knorm[tid] = kn;
-    float m = warp_max(s_val);
+  }
+
+  // ---- 4. per token (thread = token): |k|^2, anchor score, softmax weight
+  const int ti = tok[tid];
+  float s_val = -INFINITY, kn = 0.f;
+  if (ti >= 0) {
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < CPR; ++c) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(kt + (c >> 3) * L::KV_BOX + swz128(tid, c & 7));
+      const unsigned w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float x0 = bf16_lo(w[e]), x1 = bf16_hi(w[e]);
+        dot = fmaf(x0, qf[c * 8 + 2 * e], dot);
+        dot = fmaf(x1, qf[c * 8 + 2 * e + 1], dot);
+        kn = fmaf(x0, x0, kn);
+        kn = fmaf(x1, x1, kn);
+      }
+    }
+    s_val = isret[tid] ? srow[ti - p.n_sink] : dot * p.scale;
+  }
+  {
+    const float m = warp_max(s_val);
     if (lane == 0) misc[warp] = m;
   }
   __syncthreads();
-  const float m_slice = fmaxf(misc[0], misc[1]);
-  if (tid < kSlice) {
-    const float w = tok[tid] >= 0 ? expf(sc[tid] - m_slice) : 0.f;
-    wgt[tid] = w;
-    zt[tid] = 0.f;
-  }
+  const float m_slice = fmaxf(fmaxf(misc[0], misc[1]), fmaxf(misc[2], misc[3]));
+  const float w_t = ti >= 0 ? expf(s_val - m_slice) : 0.f;
+  wgt[tid] = w_t;
 
-  // ---- 4. z_i = <phi_q, phi_k(k_i)> for the retrieved rows of the slice
-  if (do_phi) {
-    constexpr int NG = kExThreads / R;       // token groups
-    constexpr int TPG = kSlice / NG;         // tokens per group
-    const int j = tid % R, tg = tid / R, t0 = tg * TPG;
-    float acc[TPG];
+  // ---- 5. z_t = <phi_q, phi_k(k_t)> from the accumulator row of this token
+  float z_t = 0.f;
+  if (has_ret) {
+    ok = mbar_wait(&bars[1], 0, s_abort);
+    ok = __syncthreads_and(ok ? 1 : 0) != 0;
+    if (ok) {
+      tc_fence_after_sync();
+      const uint32_t tmem_d = *s_tmem;
+      const float shift = -p.gamma_k * kn;
 #pragma unroll
-    for (int t = 0; t < TPG; ++t) acc[t] = 0.f;
-    for (int c = 0; c < D; ++c) {
-      const float w = Wt[c * L::WT_LD + j];
-      const float4* kp = reinterpret_cast<const float4*>(kf + c * kSlice + t0);
+      for (int c4 = 0; c4 < R / 32; ++c4) {
+        float v[32];
+        tmem_ld_x32(tmem_addr(tmem_d, warp * 32, c4 * 32), v);
+        tc_wait_ld();
 #pragma unroll
-      for (int t4 = 0; t4 < TPG / 4; ++t4) {
-        const float4 kv = kp[t4];
-        acc[4 * t4 + 0] = fmaf(w, kv.x, acc[4 * t4 + 0]);
-        acc[4 * t4 + 1] = fmaf(w, kv.y, acc[4 * t4 + 1]);
-        acc[4 * t4 + 2] = fmaf(w, kv.z, acc[4 * t4 + 2]);
-        acc[4 * t4 + 3] = fmaf(w, kv.w, acc[4 * t4 + 3]);
+        for (int j = 0; j < 32; ++j) z_t = fmaf(phiq[c4 * 32 + j], __expf(v[j] + bk[c4 * 32 + j] + shift), z_t);
       }
-    }
-    const float bj = p.b_k[(size_t)kvh * R + j], pq = phiq[j];
-    // warp w of the group covers features 32*(w in group)..; sum over the warp,
-    // then over the group's warps in fixed order
-    const int wg = (tid % R) >> 5;           // warp within the group
-#pragma unroll
-    for (int t = 0; t < TPG; ++t) {
-      float z = 0.f;
-      if (isret[t0 + t]) z = pq * expf(acc[t] + bj - p.gamma_k * knorm[t0 + t]);
-      z = warp_sum(z);
-      if (lane == 0) zpart[wg * kSlice + t0 + t] = z;
-    }
-    __syncthreads();
-    if (tid < kSlice) {
-      float z = 0.f;
-#pragma unroll
-      for (int w = 0; w < R / 32; ++w) z += zpart[w * kSlice + tid];
-      zt[tid] = z;
+      if (!isret[tid]) z_t = 0.f;
     }
   }
+  zt[tid] = z_t;
   __syncthreads();
 
-  // ---- 5. slice partials: nu = sum w_t v_t, zv = sum z_t v_t, Z = sum w_t, zs = sum z_t
+  // ---- 6. slice partials: nu = sum w_t v_t, zv = sum z_t v_t, Z = sum w_t, zs = sum z_t
   {
-    constexpr int NGV = kExThreads / D;      // token groups for the value pass (2 or 4)
+    constexpr int NGV = kExThreads / D;      // token groups for the value pass (1 or 2)
     constexpr int TPV = kSlice / NGV;
     const int dv = tid % D, tg = tid / D;
+    const unsigned char* vcol = vt + (dv >> 6) * L::KV_BOX + (dv & 7) * 2;
+    const uint32_t ch = (dv & 63) >> 3;
     float nu = 0.f, zv = 0.f;
+#pragma unroll 8
     for (int t = tg * TPV; t < (tg + 1) * TPV; ++t) {
-      const float x = __bfloat162float(vs[t * D + dv]);
+      const unsigned short raw = *reinterpret_cast<const unsigned short*>(vcol + swz128(t, ch));
+      const float x = __uint_as_float((unsigned)raw << 16);
       nu = fmaf(wgt[t], x, nu);
       zv = fmaf(zt[t], x, zv);
     }
@@ -202,18 +239,31 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   }
   __syncthreads();
   float* part = p.partials + ((size_t)row * p.max_slices + slice) * p.partial_stride;
-  if (tid < 2 * D) {
+  for (int i = tid; i < 2 * D; i += kExThreads) {
     constexpr int NGV = kExThreads / D;
-    float x = 0.f;
-#pragma unroll
-    for (int g = 0; g < NGV; ++g) x += red[g * 2 * D + tid];
-    part[4 + tid] = x;
+    float x = red[i];
+    if (NGV == 2) x += red[2 * D + i];       // second token group, fixed order
+    part[4 + i] = x;
   }
   if (tid < 32) {
-    float Z = wgt[tid] + wgt[tid + 32], zs = zt[tid] + zt[tid + 32];
+    float Z = 0.f, zs = 0.f;
+#pragma unroll
+    for (int i = 0; i < kSlice / 32; ++i) { Z += wgt[tid + 32 * i]; zs += zt[tid + 32 * i]; }
     Z = warp_sum(Z);
     zs = warp_sum(zs);
     if (tid == 0) { part[0] = m_slice; part[1] = Z; part[2] = zs; part[3] = 0.f; }
+  }
+
+  // ---- tensor memory is no longer needed
+  tc_fence_before_sync();
+  __syncthreads();
+  if (has_ret && warp == 0) {
+    tc_fence_after_sync();
+    tmem_dealloc(*s_tmem, R);
+  }
+  if (*s_abort) {
+    if (tid == 0) atomicExch(p.status, kStatusTimeout);
+    return;
   }
 
   // ---- ticket: the last slice CTA of this head merges

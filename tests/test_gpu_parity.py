@@ -76,8 +76,16 @@ def _check_decode(gl, step, frac, S, u, with_phi=True, flags=0, heads=None, topk
                     assert abs(dbg[0] - res.m_E) <= PU.ME_TOL * max(1.0, abs(res.m_E)), (b, hq, dbg[0], res.m_E)
                     assert abs(dbg[1] - res.Z_E) <= 1e-4 * res.Z_E
                 if check_resid and not res.clamped and math.isfinite(dbg[2]):
-                    assert abs(dbg[2] - res.log_Zhat_R) <= PU.LOGZ_TOL, (b, hq, dbg[2], res.log_Zhat_R)
-                    assert PU.max_rel(dbg[4:], res.y_R_hat) <= PU.Y_TOL, (b, hq)
+                    # Z_hat_R = phi_q.u_M - sum z_i is a difference (Eq. subtraction): its error is
+                    # bounded relative to the unsubtracted mass phi_q.u_M, not to what is left of it
+                    log_ZM = O.topkphi_attention(q64, K, V, inp.n_sink, inp.n_tail, kk, *_phi_arrays(phi, hq, kvh),
+                                                 S=Sh[b, kvh], u=uh[b, kvh], retrieved=ret,
+                                                 subtract=False).log_Zhat_R
+                    left = math.exp(res.log_Zhat_R - log_ZM)          # share of the mass that is left
+                    assert abs(math.exp(dbg[2] - log_ZM) - left) <= PU.LOGZ_TOL, (b, hq, dbg[2], res.log_Zhat_R)
+                    if left > 0.05:
+                        assert abs(dbg[2] - res.log_Zhat_R) <= PU.LOGZ_TOL / left, (b, hq, dbg[2], res.log_Zhat_R)
+                        assert PU.max_rel(dbg[4:], res.y_R_hat) <= PU.Y_TOL / left, (b, hq)
             else:
                 y0, _ = O.topk_attention(q64, K, V, inp.n_sink, inp.n_tail, kk, retrieved=ret)
             e = PU.max_rel(out["y"][b, hq], y0)
