@@ -251,9 +251,9 @@ def run_ours(args, rank, world, device):
         "gen_s": t_gen,
     }
     if kt is not None:
-        dom = kt["score_hist"]
+        dom = kt["score"]
         a = ab["key_stream_per_layer"] / (dom["avg_ms"] * 1e-3) / 1e9
-        out["roofline"] = {"bound": "hbm", "kernel": "score_hist_kernel", "achieved": a, "peak": peak,
+        out["roofline"] = {"bound": "hbm", "kernel": "score_kernel", "achieved": a, "peak": peak,
                            "unit": "GB/s", "frac": a / peak, "traffic": None, "peak_kind": peak_kind,
                            "avg_launch_us": dom["avg_ms"] * 1e3}
         out["kernels_us_per_launch"] = {k: v["avg_ms"] * 1e3 for k, v in kt.items()}

@@ -70,7 +70,7 @@ enum {
  * cu_seqlens[b] .. cu_seqlens[b+1]-1; its prefill length is L_b = cu_seqlens[b+1]
  * - cu_seqlens[b] >= 1.  Element (head h, row t, dim c) of k is at
  * k + h*kv_stride_head + t*kv_stride_token + c (in bf16 elements); v uses the
- * same strides.  Requirements: head_dim in {64, 128}; n_q_heads a multiple of
+ * same strides.  Requirements: 1 <= batch <= 1024; head_dim in {64, 128}; n_q_heads a multiple of
  * n_kv_heads with group size <= 8; n_feat in {64, 128}; k and v 16-byte aligned;
  * both strides multiples of 8 elements; kv_stride_token >= head_dim; total rows
  * < 2^31.  Query head h_q uses KV head h_q / (n_q_heads / n_kv_heads).
@@ -204,13 +204,14 @@ tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32
  * two host arrays of TKPHI_KERNEL_KINDS entries, and clears the record.
  */
 enum {
-  TKPHI_KERNEL_SCORE_HIST = 0,      /* key scoring + histogram (streams the mid-region keys) */
+  TKPHI_KERNEL_SCORE = 0,           /* key scoring (streams the mid-region keys) */
   TKPHI_KERNEL_COMPACT = 1,         /* bitmap and candidate lists against the threshold bin; phi_q; W_k split */
   TKPHI_KERNEL_FINALIZE_SELECT = 2, /* exact threshold, ties, ascending index list */
   TKPHI_KERNEL_EXACT_RESIDUAL = 3,  /* exact branch, subtraction, residual, merge */
   TKPHI_KERNEL_BUILD = 4,           /* prefill summary build */
   TKPHI_KERNEL_MEMSET = 5,          /* clearing counters and histograms */
-  TKPHI_KERNEL_KINDS = 6
+  TKPHI_KERNEL_HIST = 6,            /* score histogram and threshold bin */
+  TKPHI_KERNEL_KINDS = 7
 };
 void tkphi_kernel_timing_enable(int32_t on);
 tkphi_status tkphi_kernel_timing_read(float* ms_out, int32_t* count_out);

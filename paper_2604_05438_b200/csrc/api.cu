@@ -107,11 +107,9 @@ int n_sm_cached() {
 }
 
 void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, WsLayout* L) {
-  const int passes = (kv->n_q_heads / kv->n_kv_heads + 3) / 4;
   size_t o = 0;
-  L->passes = passes;
   L->status = o;        o += 256;
-  L->unit_counter = o;  o = align_up(o + sizeof(unsigned) * sh.units * passes, 256);
+  L->unit_counter = o;  o = align_up(o + sizeof(unsigned) * sh.rows, 256);
   L->row_counter = o;   o = align_up(o + sizeof(unsigned) * sh.rows, 256);
   L->hist = o;          o = align_up(o + sizeof(unsigned) * (size_t)sh.rows * kHistBins, 256);
   L->zero_end = o;
@@ -289,11 +287,16 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
     st = make_key_tensor_map(kv, sh.total_tokens, &tm);
     if (st != TKPHI_OK) return st;
     long long grid = sh.score_tiles < n_sm_cached() ? sh.score_tiles : n_sm_cached();
-    for (int pass = 0; pass < L.passes; ++pass) {
-      ScopedSpan sp(cs, TKPHI_KERNEL_SCORE_HIST);
-      e = launch_score_hist(p, tm, pass, (int)grid, cs);
-      if (e != cudaSuccess) return cuda_fail(e, "score_hist launch");
+    {
+      ScopedSpan sp(cs, TKPHI_KERNEL_SCORE);
+      e = launch_score(p, tm, (int)grid, cs);
     }
+    if (e != cudaSuccess) return cuda_fail(e, "score launch");
+    {
+      ScopedSpan sp(cs, TKPHI_KERNEL_HIST);
+      e = launch_hist(p, sh.max_mid, cs);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "hist launch");
   }
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_COMPACT);

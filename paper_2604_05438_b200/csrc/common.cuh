@@ -13,7 +13,7 @@ namespace tkphi {
 constexpr int kHistBits = 12;                 // leading bits of the ordered score key
 constexpr int kHistBins = 1 << kHistBits;     // bins of the fused first-pass histogram
 constexpr int kLowBits = 32 - kHistBits;      // bits refined inside the threshold bin
-constexpr int kMaxBatch = 4096;               // sequences per call
+constexpr int kMaxBatch = 1024;               // sequences per call
 constexpr int kSlice = 128;                   // exact-support tokens per CTA of the exact/residual kernel (= MMA M)
 constexpr int kCompactChunk = 4096;           // scores per CTA of the compaction kernel
 constexpr int kMaxChunks = 2048;              // compaction chunks per sequence the selection kernel can index
@@ -43,7 +43,7 @@ struct Problem {
   int with_phi;                    // 0: selection-only, 1: Top-K+phi
   // workspace pieces (device pointers)
   int* status;
-  unsigned* unit_counter;          // [batch*n_kv_heads*passes]
+  unsigned* unit_counter;          // [batch*n_q_heads] histogram-chunk tickets
   unsigned* row_counter;           // [batch*n_q_heads]
   int4* rowinfo;                   // [rows]: x = threshold bin, y = count above, z = count in bin
   unsigned* hist;                  // [rows][kHistBins]
@@ -79,7 +79,7 @@ struct BuildProblem {
 struct WsLayout {
   size_t status, unit_counter, row_counter, hist, zero_end;
   size_t rowinfo, scores, bm_sure, cand, chunk_ncand, wk_img, idx, aq, partials, total;
-  int max_slices, partial_stride, passes, max_chunks;
+  int max_slices, partial_stride, max_chunks;
   // build
   size_t b_partials; int chunk_len, chunks_per_unit;
 };
@@ -162,7 +162,8 @@ __device__ __forceinline__ long long bitmap_row_base(const Problem& p, int b, in
 
 // ---------------------------------------------------------------- host launchers
 // Each returns cudaGetLastError() after enqueuing on `stream`.
-cudaError_t launch_score_hist(const Problem& p, const CUtensorMap& tmap_k, int pass, int n_sm, cudaStream_t stream);
+cudaError_t launch_score(const Problem& p, const CUtensorMap& tmap_k, int n_sm, cudaStream_t stream);
+cudaError_t launch_hist(const Problem& p, int max_mid, cudaStream_t stream);
 cudaError_t launch_compact(const Problem& p, int max_mid, cudaStream_t stream);
 cudaError_t launch_finalize_select(const Problem& p, cudaStream_t stream);
 cudaError_t launch_exact_residual(const Problem& p, cudaStream_t stream);

@@ -152,16 +152,14 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
       tc_fence_after_sync();
       constexpr uint32_t idesc = umma_idesc_bf16(128, R, 0, 0);
       const uint32_t tmem_d = *s_tmem;
-      const uint32_t ka = smem_u32(kt);
+      const uint64_t adesc0 = umma_smem_desc(smem_u32(kt), 16, 1024);
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        const uint32_t wa = smem_u32(half == 0 ? whi : wlo);
+        const uint64_t bdesc0 = umma_smem_desc(smem_u32(half == 0 ? whi : wlo), 16, 1024);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint64_t adesc = umma_smem_desc(ka + (k >> 2) * L::KV_BOX + (k & 3) * 32, 16, 1024);
-          const uint64_t bdesc = umma_smem_desc(wa + (k >> 2) * L::W_BOX + (k & 3) * 32, 16, 1024);
-          umma_ss(tmem_d, adesc, bdesc, idesc, (half | k) ? 1u : 0u);
-        }
+        for (int k = 0; k < D / 16; ++k)
+          umma_ss(tmem_d, adesc0 + (uint64_t)(((k >> 2) * L::KV_BOX + (k & 3) * 32) >> 4),
+                  bdesc0 + (uint64_t)(((k >> 2) * L::W_BOX + (k & 3) * 32) >> 4), idesc, (half | k) ? 1u : 0u);
       }
       tc_commit(&bars[1]);
     }

@@ -3,17 +3,17 @@
 // and select, per query head, the K highest-scoring mid-region indices with ties
 // broken towards the lower index (exhaustive Top-K control selector, Sec. 5.1).
 //
-// Three kernels:
-//   score_hist_kernel      streams the keys once.  A producer thread issues TMA loads of
-//                          128B-swizzled 32 KB key tiles into a 4-stage mbarrier ring; one
-//                          thread issues tcgen05.mma with the key tile as the A operand
-//                          straight from shared memory and the group's queries (zero padded
-//                          to 16 rows) as B, so the dot products cost no issue slots of the
-//                          CUDA cores; four warps read the 128 x 16 fp32 accumulators back
-//                          from tensor memory, write the score rows and add to a 4096-bin
-//                          histogram of the leading 12 bits of the order-preserving score
-//                          key.  The last CTA to finish a (sequence, KV head) unit turns the
-//                          histogram into a threshold bin per query head.
+// Four kernels:
+//   score_kernel           streams the keys once.  A producer thread issues TMA loads of
+//                          128B-swizzled 32 KB key tiles into a 6-stage mbarrier ring; one
+//                          thread issues tcgen05.mma with the key tile as an operand straight
+//                          from shared memory and the group's queries (zero padded) as the
+//                          other, so the dot products cost no issue slots of the CUDA cores;
+//                          one warp reads the fp32 accumulators back from tensor memory and
+//                          writes the score rows.
+//   hist_kernel            one pass over the (L2-resident) scores: 4096-bin histogram of the
+//                          leading 12 bits of the order-preserving score key per query head;
+//                          the last CTA of a head turns it into a threshold bin.
 //   compact_kernel         one pass over the (L2-resident) scores: a bitmap of positions above
 //                          the threshold bin and, per 4096-score chunk, the ordered list of
 //                          positions inside it.  Spare CTAs evaluate the query-side
@@ -27,22 +27,21 @@
 
 namespace tkphi {
 
-// ------------------------------------------------------------------ score + histogram
-constexpr int kScoreThreads = 192;        // warp 0: TMA producer, warp 1: MMA issuer, warps 2..5: read-back
-constexpr int kScoreStages = 4;
+// ------------------------------------------------------------------ scoring
+constexpr int kScoreThreads = 96;         // warp 0: read-back, warp 1: MMA issuer, warp 2: TMA producer
+constexpr int kScoreStages = 6;
 constexpr int kScoreTileBytes = 32768;
-constexpr int kAccStages = 4;             // accumulator buffers in tensor memory
-constexpr int kScoreN = 16;               // MMA N: query heads of the group, zero padded
-constexpr int kEpiThreads = 128;
+constexpr int kScoreM = 64;               // MMA M: query heads of the group (<= 8), zero padded
+constexpr int kTmemCols = 512;
 
 template <int D>
 struct ScoreCfg {
-  static constexpr int TK = kScoreTileBytes / (2 * D);   // keys per TMA tile
-  static constexpr int SUB = TK / 128;                   // 128-key MMA tiles per TMA tile
+  static constexpr int TK = kScoreTileBytes / (2 * D);   // keys per TMA tile = MMA N (128 or 256)
   static constexpr int BOXES = D / 64;                   // 64-dim (128-byte) column blocks
   static constexpr int BOX_BYTES = TK * 128;
-  static constexpr int QBOX_BYTES = kScoreN * 128;
-  static_assert(TK * D * 2 == kScoreTileBytes && SUB >= 1, "tile size");
+  static constexpr int QBOX_BYTES = kScoreM * 128;
+  static constexpr int ACC_STAGES = kTmemCols / TK;      // accumulator buffers in tensor memory
+  static_assert(TK * D * 2 == kScoreTileBytes && TK <= 256, "tile size");
 };
 
 struct TileCursor {
@@ -75,69 +74,32 @@ __device__ __forceinline__ void cursor_next(TileCursor& c, const int* pre, int b
   } while (c.nt == 0);
 }
 
-__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// True iff `x` holds on all 128 read-back threads (a barrier among them).
-__device__ __forceinline__ bool epi_all(bool x) {
-  uint32_t r;
-  asm volatile(
-      "{\n"
-      " .reg .pred p, q;\n"
-      " setp.ne.b32 q, %1, 0;\n"
-      " bar.red.and.pred p, 1, 128, q;\n"
-      " selp.b32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(r)
-      : "r"(x ? 1u : 0u)
-      : "memory");
-  return r != 0;
-}
-
-// Exclusive prefix sum over the 128 read-back threads (et = 0..127); scratch >= 8 ints.
-__device__ __forceinline__ int epi_exclusive_scan(int x, int et, int* scratch, int* total) {
-  const int lane = et & 31, w = et >> 5;
-  int incl = x;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
-  }
-  epi_sync();
-  if (lane == 31) scratch[w] = incl;
-  epi_sync();
-  int base = 0, tot = 0;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int s = scratch[i];
-    if (i < w) base += s;
-    tot += s;
-  }
-  *total = tot;
-  return base + incl - x;
-}
-
-template <int D, int G>
+// The contraction is issued as scores^T = Q K^T: the group's queries (zero padded to 64
+// rows) are the A operand and the key tile, exactly as TMA lands it, is the B operand
+// (N = keys of the tile).  The tensor core fetches B rows twice as fast as A rows, which
+// halves the time the key tile is being read out of shared memory compared with the
+// transposed form; row g of the accumulator (tensor-memory lane g) holds head g's scores.
+template <int D>
 __global__ void __launch_bounds__(kScoreThreads, 1)
-score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, const int g0, const int pass) {
+score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
   using C = ScoreCfg<D>;
-  constexpr int TK = C::TK, SUB = C::SUB, BOXES = C::BOXES;
+  constexpr int TK = C::TK, BOXES = C::BOXES, ACC = C::ACC_STAGES;
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* tiles = smem;                                              // [stages][32 KB]
-  unsigned char* qtile = smem + kScoreStages * kScoreTileBytes;             // [BOXES][16 rows][128 B]
-  unsigned* hist_s = reinterpret_cast<unsigned*>(qtile + BOXES * C::QBOX_BYTES);   // [G][bins]
-  int* pre = reinterpret_cast<int*>(hist_s + G * kHistBins);               // [batch+1]
+  unsigned char* qtile = smem + kScoreStages * kScoreTileBytes;             // [BOXES][64 rows][128 B]
+  int* pre = reinterpret_cast<int*>(qtile + BOXES * C::QBOX_BYTES);        // [batch+1]
   uint64_t* bars = reinterpret_cast<uint64_t*>(pre + kMaxBatch + 2);
   uint64_t* full = bars;                          // TMA tile landed
   uint64_t* empty = full + kScoreStages;          // MMAs that read the tile are done
   uint64_t* acc_full = empty + kScoreStages;      // accumulator buffer holds a finished tile
-  uint64_t* acc_empty = acc_full + kAccStages;    // accumulator buffer has been read back
-  uint64_t* qbar = acc_empty + kAccStages;        // every MMA issued so far is done
+  uint64_t* acc_empty = acc_full + ACC;           // accumulator buffer has been read back
+  uint64_t* qbar = acc_empty + ACC;               // every MMA issued so far is done
   int* scratch = reinterpret_cast<int*>(qbar + 1);                         // [40]
-  int* s_flag = scratch + 36;
   volatile int* s_abort = scratch + 37;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(scratch + 38);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n_kv = p.n_kv_heads, batch = p.batch;
+  const int n_kv = p.n_kv_heads, batch = p.batch, G = p.group;
 
   // ---- tiles per sequence -> prefix in shared memory
   {
@@ -166,15 +128,14 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
     }
     if (tid == 0) pre[batch] = total;
   }
-  for (int i = tid; i < G * kHistBins; i += kScoreThreads) hist_s[i] = 0;
   if (tid == 0) {
     for (int s = 0; s < kScoreStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < kAccStages; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kEpiThreads); }
+    for (int a = 0; a < ACC; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 1); }
     mbar_init(qbar, 1);
     mbar_fence_init();
     *s_abort = 0;
   }
-  if (warp == 1) tmem_alloc(s_tmem, kAccStages * kScoreN);
+  if (warp == 1) tmem_alloc(s_tmem, kTmemCols);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -185,18 +146,19 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
   const int n_my = f1 - f0;
 
   if (n_my > 0) {
-    if (warp == 0) {
+    if (warp == 2) {
       // ================================================================ TMA producer
       if (lane == 0) {
         TileCursor pc;
         cursor_seek(pc, pre, batch, n_kv, f0);
-        int it = 0;
+        int it = 0, row_b = -1, row0 = 0;
         for (; it < n_my; ++it) {
           const int slot = it % kScoreStages;
           const uint32_t ph = (uint32_t)(it / kScoreStages) & 1u;
           if (!mbar_wait(&empty[slot], ph ^ 1u, s_abort)) break;
           mbar_expect_tx(&full[slot], kScoreTileBytes);
-          const int row = (int)(p.cu_seqlens[pc.b] + p.n_sink) + pc.t * TK;
+          if (pc.b != row_b) { row_b = pc.b; row0 = (int)(p.cu_seqlens[pc.b] + p.n_sink); }
+          const int row = row0 + pc.t * TK;
 #pragma unroll
           for (int x = 0; x < BOXES; ++x)
             tma_load_3d(tiles + slot * kScoreTileBytes + x * C::BOX_BYTES, &tmap_k, &full[slot], x * 64, row,
@@ -218,10 +180,14 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
       }
     } else if (warp == 1) {
       // ================================================================ MMA issuer
-      constexpr uint32_t idesc = umma_idesc_bf16(128, kScoreN, 0, 0);
+      constexpr uint32_t idesc = umma_idesc_bf16(kScoreM, TK, 0, 0);
+      // operand descriptors: the address field counts 16-byte units, so moving to another
+      // tile, column block or K step is one 64-bit add of a small constant
+      const uint64_t adesc0 = umma_smem_desc(smem_u32(qtile), 16, 1024);
+      const uint64_t bdesc0 = umma_smem_desc(smem_u32(tiles), 16, 1024);
       TileCursor mc;
       cursor_seek(mc, pre, batch, n_kv, f0);
-      int cur_b = -1, cur_kvh = -1, acc_it = 0;
+      int cur_b = -1, cur_kvh = -1;
       uint32_t qphase = 0;
       bool ok = true;
       for (int it = 0; it < n_my && ok; ++it) {
@@ -230,15 +196,14 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
           if (it > 0) {
             if (lane == 0) tc_commit(qbar);
             __syncwarp();
-            ok = mbar_wait(qbar, qphase, s_abort);
+            ok = __all_sync(0xffffffffu, mbar_wait(qbar, qphase, s_abort));
             qphase ^= 1u;
-            ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
           }
           cur_b = mc.b; cur_kvh = mc.kvh;
-          // rows 0..G-1: the group's queries, rows G..15 zero; 128B-swizzled like the key tiles
-          const __nv_bfloat16* qp = p.q + ((size_t)cur_b * p.n_q_heads + cur_kvh * p.group + g0) * D;
-          for (int i = lane; i < kScoreN * (D / 8); i += 32) {
+          // rows 0..G-1: the group's queries, rows G..63 zero; 128B-swizzled like the key tiles
+          const __nv_bfloat16* qp = p.q + ((size_t)cur_b * p.n_q_heads + cur_kvh * G) * D;
+          for (int i = lane; i < kScoreM * (D / 8); i += 32) {
             const int r = i / (D / 8), c = i % (D / 8);
             uint4 val = make_uint4(0, 0, 0, 0);
             if (r < G) val = *reinterpret_cast<const uint4*>(qp + (size_t)r * D + c * 8);
@@ -247,129 +212,71 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
           fence_proxy_async_smem();
           __syncwarp();
         }
-        const int slot = it % kScoreStages;
-        const uint32_t ph = (uint32_t)(it / kScoreStages) & 1u;
         if (lane == 0) {
-          ok = mbar_wait(&full[slot], ph, s_abort);
-          tc_fence_after_sync();
-          for (int sub = 0; sub < SUB && ok; ++sub, ++acc_it) {
-            const int a = acc_it % kAccStages;
-            const uint32_t aph = (uint32_t)(acc_it / kAccStages) & 1u;
-            ok = mbar_wait(&acc_empty[a], aph ^ 1u, s_abort);
-            if (!ok) break;
+          const int slot = it % kScoreStages;
+          const uint32_t ph = (uint32_t)(it / kScoreStages) & 1u;
+          const int a = it % ACC;
+          const uint32_t aph = (uint32_t)(it / ACC) & 1u;
+          ok = mbar_wait(&full[slot], ph, s_abort) && mbar_wait(&acc_empty[a], aph ^ 1u, s_abort);
+          if (ok) {
             tc_fence_after_sync();
-            const uint32_t tile_addr = smem_u32(tiles + slot * kScoreTileBytes) + sub * (128 * 128);
-            const uint32_t q_addr = smem_u32(qtile);
+            const uint64_t bdesc = bdesc0 + (uint64_t)((slot * kScoreTileBytes) >> 4);
 #pragma unroll
-            for (int k = 0; k < D / 16; ++k) {
-              const uint64_t adesc = umma_smem_desc(tile_addr + (k >> 2) * C::BOX_BYTES + (k & 3) * 32, 16, 1024);
-              const uint64_t bdesc = umma_smem_desc(q_addr + (k >> 2) * C::QBOX_BYTES + (k & 3) * 32, 16, 1024);
-              umma_ss(tmem_base + a * kScoreN, adesc, bdesc, idesc, k > 0 ? 1u : 0u);
-            }
+            for (int k = 0; k < D / 16; ++k)
+              umma_ss(tmem_base + a * TK, adesc0 + (uint64_t)(((k >> 2) * C::QBOX_BYTES + (k & 3) * 32) >> 4),
+                      bdesc + (uint64_t)(((k >> 2) * C::BOX_BYTES + (k & 3) * 32) >> 4), idesc, k > 0 ? 1u : 0u);
             tc_commit(&acc_full[a]);
+            tc_commit(&empty[slot]);
           }
-          if (ok) tc_commit(&empty[slot]);
         }
-        acc_it = __shfl_sync(0xffffffffu, acc_it, 0);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         cursor_next(mc, pre, batch, n_kv);
       }
     } else {
-      // ================================================================ read-back, scores, histogram
-      const int et = tid - 64;                  // 0..127
-      const int quad = warp & 3;                // tensor-memory lane quadrant this warp may read
-      const int krow = quad * 32 + lane;        // key row inside a 128-key MMA tile
+      // ================================================================ read-back, score rows
+      // warp 0 reads tensor-memory lanes 0..15: thread t holds head (t / 4), key columns
+      // 8 i + 2 (t % 4) + {0, 1} of each 8-column block i (the second register pair of a
+      // block belongs to rows 8..15, which are zero padding)
       TileCursor cc;
       cursor_seek(cc, pre, batch, n_kv, f0);
-      int cur_b = -1, cur_kvh = -1, tiles_done = 0, n_mid = 0, acc_it = 0;
-      long long row_base0 = 0, len_b = 0;
+      int cur_b = -1, cur_kvh = -1, n_mid = 0;
+      long long len_b = 0;
+      float* my_row = nullptr;
+      const int g = lane >> 2, cpair = 2 * (lane & 3);
       bool ok = true;
-
-      auto finish_unit = [&]() {
-        // publish this CTA's share of the unit's histogram, then take a ticket
-        epi_sync();
-        const int row0 = cur_b * p.n_q_heads + cur_kvh * p.group + g0;
-        for (int i = et; i < G * kHistBins; i += kEpiThreads) {
-          unsigned h = hist_s[i];
-          if (h) {
-            atomicAdd(&p.hist[(size_t)(row0 + i / kHistBins) * kHistBins + (i % kHistBins)], h);
-            hist_s[i] = 0;
-          }
-        }
-        __threadfence();
-        epi_sync();
-        if (et == 0) {
-          const int unit = cur_b * n_kv + cur_kvh;
-          const unsigned nt_unit = (unsigned)((pre[cur_b + 1] - pre[cur_b]) / n_kv);
-          unsigned prev = atomicAdd(&p.unit_counter[(size_t)pass * batch * n_kv + unit], (unsigned)tiles_done);
-          *s_flag = (prev + (unsigned)tiles_done == nt_unit) ? 1 : 0;
-        }
-        epi_sync();
-        if (*s_flag) {
-          // last CTA of the unit: threshold bin per query head from the full histogram
-          __threadfence();
-          const int K = p.topk[cur_b];
-          constexpr int BPT = kHistBins / kEpiThreads;       // 32 bins per thread
-          for (int g = 0; g < G; ++g) {
-            const unsigned* h = p.hist + (size_t)(row0 + g) * kHistBins + et * BPT;
-            unsigned loc[BPT];
-            int lsum = 0;
-#pragma unroll
-            for (int i = 0; i < BPT; ++i) { loc[i] = __ldcg(h + i); lsum += (int)loc[i]; }
-            int total;
-            int excl = epi_exclusive_scan(lsum, et, scratch, &total);
-            int above = total - excl - lsum;          // elements in bins above this thread's range
-            if (above < K && K <= above + lsum) {
-              int cum = above;
-#pragma unroll
-              for (int i = BPT - 1; i >= 0; --i) {
-                if (cum < K && K <= cum + (int)loc[i])
-                  p.rowinfo[row0 + g] = make_int4(et * BPT + i, cum, (int)loc[i], total);
-                cum += (int)loc[i];
-              }
-            }
-          }
-        }
-        epi_sync();
-        tiles_done = 0;
-      };
-
       for (int it = 0; it < n_my && ok; ++it) {
         if (cc.b != cur_b || cc.kvh != cur_kvh) {
-          if (cur_b >= 0) finish_unit();
           cur_b = cc.b; cur_kvh = cc.kvh;
           const long long cu_b = p.cu_seqlens[cur_b];
           len_b = p.cu_seqlens[cur_b + 1] - cu_b;
           n_mid = mid_len(len_b, p.n_sink, p.n_tail);
-          row_base0 = score_row_base(p, cur_b, cur_kvh * p.group + g0, cu_b, len_b);
+          my_row = p.scores + score_row_base(p, cur_b, cur_kvh * G, cu_b, len_b) + (long long)g * len_b;
         }
-        for (int sub = 0; sub < SUB; ++sub, ++acc_it) {
-          const int a = acc_it % kAccStages;
-          const uint32_t aph = (uint32_t)(acc_it / kAccStages) & 1u;
-          ok = epi_all(mbar_wait(&acc_full[a], aph, s_abort));   // all 128 threads go on, or none
-          if (!ok) break;
-          tc_fence_after_sync();
-          float v[4];
-          tmem_ld_x4(tmem_addr(tmem_base, quad * 32, a * kScoreN), v);
-          tc_wait_ld();
-          tc_fence_before_sync();
-          mbar_arrive(&acc_empty[a]);
-          const int j = cc.t * TK + sub * 128 + krow;
-          if (j < n_mid) {
+        const int a = it % ACC;
+        const uint32_t aph = (uint32_t)(it / ACC) & 1u;
+        ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[a], aph, s_abort));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int j0 = cc.t * TK + cpair;
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-              const float sc = v[g] * p.scale;
-              p.scores[row_base0 + (long long)g * len_b + j] = sc;
-              atomicAdd(&hist_s[g * kHistBins + (ordered_key(sc) >> kLowBits)], 1u);
+        for (int half = 0; half < TK / 64; ++half) {
+          float v[32];
+          tmem_ld_16x256b_x8(tmem_addr(tmem_base, 0, a * TK + half * 64), v);
+          tc_wait_ld();
+          if (g < G) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int j = j0 + half * 64 + i * 8;
+              if (j < n_mid) my_row[j] = v[4 * i] * p.scale;
+              if (j + 1 < n_mid) my_row[j + 1] = v[4 * i + 1] * p.scale;
             }
           }
         }
-        ++tiles_done;
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[a]);
         cursor_next(cc, pre, batch, n_kv);
       }
-      // a CTA that gave up publishes nothing: the unit's ticket never completes and the
-      // status word tells the host
-      if (ok) finish_unit();
     }
   }
 
@@ -379,39 +286,104 @@ score_hist_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p, c
   if (*s_abort && tid == 0) atomicExch(p.status, kStatusTimeout);
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kAccStages * kScoreN);
+    tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
-static size_t score_smem_bytes(int D, int G) {
-  return (size_t)kScoreStages * kScoreTileBytes + (size_t)(D / 64) * kScoreN * 128 + (size_t)G * kHistBins * 4 +
-         (size_t)(kMaxBatch + 2) * 4 + (2 * kScoreStages + 2 * kAccStages + 1) * 8 + 40 * 4 + 64;
+static size_t score_smem_bytes(int D) {
+  return (size_t)kScoreStages * kScoreTileBytes + (size_t)(D / 64) * kScoreM * 128 + (size_t)(kMaxBatch + 2) * 4 +
+         (2 * kScoreStages + 2 * 4 + 1) * 8 + 40 * 4 + 64;
 }
 
-template <int D, int G>
-static cudaError_t launch_score_t(const Problem& p, const CUtensorMap& tm, int g0, int pass, int n_sm,
-                                  cudaStream_t st) {
+template <int D>
+static cudaError_t launch_score_t(const Problem& p, const CUtensorMap& tm, int n_sm, cudaStream_t st) {
   static bool configured = false;   // attribute is per function; cheap to set once
-  const size_t smem = score_smem_bytes(D, G);
+  const size_t smem = score_smem_bytes(D);
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(score_hist_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(score_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  score_hist_kernel<D, G><<<n_sm, kScoreThreads, smem, st>>>(tm, p, g0, pass);
+  score_kernel<D><<<n_sm, kScoreThreads, smem, st>>>(tm, p);
   return cudaGetLastError();
 }
 
-cudaError_t launch_score_hist(const Problem& p, const CUtensorMap& tm, int pass, int n_sm, cudaStream_t st) {
-  const int g0 = pass * 4;
-  const int g = p.group - g0 < 4 ? p.group - g0 : 4;
-#define TKPHI_DISPATCH(DD, GG) \
-  if (p.head_dim == DD && g == GG) return launch_score_t<DD, GG>(p, tm, g0, pass, n_sm, st);
-  TKPHI_DISPATCH(64, 1) TKPHI_DISPATCH(64, 2) TKPHI_DISPATCH(64, 3) TKPHI_DISPATCH(64, 4)
-  TKPHI_DISPATCH(128, 1) TKPHI_DISPATCH(128, 2) TKPHI_DISPATCH(128, 3) TKPHI_DISPATCH(128, 4)
-#undef TKPHI_DISPATCH
+cudaError_t launch_score(const Problem& p, const CUtensorMap& tm, int n_sm, cudaStream_t st) {
+  if (p.head_dim == 64) return launch_score_t<64>(p, tm, n_sm, st);
+  if (p.head_dim == 128) return launch_score_t<128>(p, tm, n_sm, st);
   return cudaErrorInvalidValue;
+}
+
+// ------------------------------------------------------------------ histogram and threshold bin
+constexpr int kHistThreads = 512;
+constexpr int kHistChunk = 16384;                       // scores per CTA
+
+__global__ void __launch_bounds__(kHistThreads) hist_kernel(const Problem p) {
+  __shared__ unsigned h[kHistBins];
+  __shared__ int scratch[40];
+  __shared__ int s_last;
+  const int b = blockIdx.z, hq = blockIdx.y, tid = threadIdx.x;
+  const int row = b * p.n_q_heads + hq;
+  const int K = p.topk[b];
+  if (K == 0) return;
+  const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
+  const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
+  const int chunk0 = blockIdx.x * kHistChunk;
+  if (chunk0 >= n_mid) return;
+  const int n_chunks = (n_mid + kHistChunk - 1) / kHistChunk;
+  const float* srow = p.scores + score_row_base(p, b, hq, cu_b, len_b);
+  for (int i = tid; i < kHistBins; i += kHistThreads) h[i] = 0;
+  __syncthreads();
+  constexpr int PER = kHistChunk / kHistThreads;        // 32 scores per thread, all loads in flight
+  float sc[PER];
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const int j = chunk0 + i * kHistThreads + tid;
+    sc[i] = j < n_mid ? __ldcg(srow + j) : 0.f;
+  }
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const int j = chunk0 + i * kHistThreads + tid;
+    if (j < n_mid) atomicAdd(&h[ordered_key(sc[i]) >> kLowBits], 1u);
+  }
+  __syncthreads();
+  unsigned* gh = p.hist + (size_t)row * kHistBins;
+  for (int i = tid; i < kHistBins; i += kHistThreads) {
+    const unsigned c = h[i];
+    if (c) atomicAdd(&gh[i], c);
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&p.unit_counter[row], 1u) == (unsigned)(n_chunks - 1));
+  __syncthreads();
+  if (!s_last) return;
+  // last CTA of this query head: threshold bin from the full histogram
+  __threadfence();
+  constexpr int BPT = kHistBins / kHistThreads;         // 8 bins per thread
+  const uint4 lo = __ldcg(reinterpret_cast<const uint4*>(gh + tid * BPT));
+  const uint4 hi = __ldcg(reinterpret_cast<const uint4*>(gh + tid * BPT + 4));
+  const unsigned loc[BPT] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+  int lsum = 0;
+#pragma unroll
+  for (int i = 0; i < BPT; ++i) lsum += (int)loc[i];
+  int total;
+  const int excl = block_exclusive_scan(lsum, scratch, &total);
+  const int above = total - excl - lsum;                // elements in bins above this thread's range
+  if (above < K && K <= above + lsum) {
+    int cum = above;
+#pragma unroll
+    for (int i = BPT - 1; i >= 0; --i) {
+      if (cum < K && K <= cum + (int)loc[i]) p.rowinfo[row] = make_int4(tid * BPT + i, cum, (int)loc[i], total);
+      cum += (int)loc[i];
+    }
+  }
+}
+
+cudaError_t launch_hist(const Problem& p, int max_mid, cudaStream_t st) {
+  if (max_mid <= 0) return cudaSuccess;
+  dim3 grid((max_mid + kHistChunk - 1) / kHistChunk, p.n_q_heads, p.batch);
+  hist_kernel<<<grid, kHistThreads, 0, st>>>(p);
+  return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------ compaction against the threshold bin
