@@ -89,7 +89,8 @@ typedef struct {
   int64_t kv_stride_head, kv_stride_token; /* in elements */
 } tkphi_kv_desc;
 
-/* phi(x) = exp(W x + b - gamma ||x||^2); row-major fp32 parameters on the device. */
+/* phi(x) = exp(W x + b - gamma ||x||^2); row-major fp32 parameters on the device; w_q and
+ * w_k 16-byte aligned (as are S and u where a call takes them). */
 typedef struct {
   const float* w_q; /* [n_q_heads][n_feat][head_dim] */
   const float* b_q; /* [n_q_heads][n_feat] */

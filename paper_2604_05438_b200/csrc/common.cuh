@@ -54,7 +54,7 @@ struct Problem {
   int max_chunks;
   __nv_bfloat16* wk_img;           // [n_kv_heads][2][r*d] W_k split into bf16 hi / lo, stored as MMA operand tiles
   int* idx;                        // [rows][topk_max] ascending retrieved positions
-  float* aq;                       // [rows][n_feat + 4]: exp(a_q - m_q) per feature, then m_q
+  float* aq;                       // [rows][n_feat + head_dim + 4]: exp(a_q - m_q), m_q, w.u_M, S_M w
   float* partials;                 // [rows][max_slices][partial_stride]
   int max_slices, partial_stride;
   float scale;                     // 1/sqrt(head_dim)

@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   for (int c = tid; c < D; c += kExThreads) qf[c] = __bfloat162float(p.q[(size_t)row * D + c]);
   if (do_phi) {
     for (int j = tid; j < R; j += kExThreads) {
-      phiq[j] = p.aq[(size_t)row * (R + 4) + j];
+      phiq[j] = p.aq[(size_t)row * (R + D + 4) + j];
       bk[j] = p.b_k[(size_t)kvh * R + j];
     }
   }
@@ -275,19 +275,31 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   if (misc[8] == 0.f) return;
   __threadfence();
 
+  // slice partials are combined in slice order by a fixed assignment of slices to
+  // lanes and of output columns to threads, so the result does not depend on timing
   const float* parts = p.partials + (size_t)row * p.max_slices * p.partial_stride;
-  float m_E = -INFINITY;
+  float m_loc = -INFINITY;
   if (nE > 0)
-    for (int s = 0; s < n_slices; ++s) m_E = fmaxf(m_E, __ldcg(parts + (size_t)s * p.partial_stride));
-  float Z_E = 0.f, zs = 0.f;
-  for (int s = 0; s < n_slices; ++s) {
-    const float* ps = parts + (size_t)s * p.partial_stride;
-    const float f = nE > 0 ? expf(__ldcg(ps) - m_E) : 0.f;
-    Z_E = fmaf(f, __ldcg(ps + 1), Z_E);
-    zs += __ldcg(ps + 2);
+    for (int s = tid; s < n_slices; s += kExThreads) m_loc = fmaxf(m_loc, __ldcg(parts + (size_t)s * p.partial_stride));
+  m_loc = warp_max(m_loc);
+  if (lane == 0) misc[warp] = m_loc;
+  __syncthreads();
+  const float m_E = fmaxf(fmaxf(misc[0], misc[1]), fmaxf(misc[2], misc[3]));
+  if (warp == 0) {
+    float Zp = 0.f, zp = 0.f;
+    for (int s = lane; s < n_slices; s += 32) {
+      const float* ps = parts + (size_t)s * p.partial_stride;
+      const float f = nE > 0 ? expf(__ldcg(ps) - m_E) : 0.f;
+      Zp = fmaf(f, __ldcg(ps + 1), Zp);
+      zp += __ldcg(ps + 2);
+    }
+    Zp = warp_sum(Zp);
+    zp = warp_sum(zp);
+    if (lane == 0) { misc[4] = Zp; misc[5] = zp; }
   }
   float nu_E = 0.f, zv = 0.f;
   if (tid < D) {
+#pragma unroll 4
     for (int s = 0; s < n_slices; ++s) {
       const float* ps = parts + (size_t)s * p.partial_stride;
       const float f = nE > 0 ? expf(__ldcg(ps) - m_E) : 0.f;
@@ -295,35 +307,20 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
       zv += __ldcg(ps + 4 + D + tid);
     }
   }
+  __syncthreads();
+  const float Z_E = misc[4], zs = misc[5];
   float y = 0.f, yR = 0.f, logZR = -INFINITY, Mx = m_E;
   if (p.with_phi) {
-    // S_M phi_q and phi_q . u_M, both in units of exp(m_q)
-    for (int j = tid; j < R; j += kExThreads) phiq[j] = p.aq[(size_t)row * (R + 4) + j];
-    __syncthreads();
-    const float m_q = p.aq[(size_t)row * (R + 4) + R];
-    const float* Sg = p.S + ((size_t)b * p.n_kv_heads + kvh) * D * R;
-    const float* ug = p.u + ((size_t)b * p.n_kv_heads + kvh) * R;
-    // one warp per row of S: lanes run along the features
-    for (int dv = warp; dv < D; dv += kExThreads / 32) {
-      float a = 0.f;
-      for (int j = lane; j < R; j += 32) a = fmaf(Sg[(size_t)dv * R + j], phiq[j], a);
-      a = warp_sum(a);
-      if (lane == 0) red[dv] = a;
-    }
-    if (warp == 0) {
-      float a = 0.f;
-      for (int j = lane; j < R; j += 32) a = fmaf(ug[j], phiq[j], a);
-      a = warp_sum(a);
-      if (lane == 0) misc[9] = a;
-    }
-    __syncthreads();
-    const float Zt = misc[9] - zs;                         // Z_hat_R / exp(m_q)
+    // S_M phi_q and phi_q . u_M (in units of exp(m_q)) were prepared alongside phi_q
+    const float* aqr = p.aq + (size_t)row * (R + D + 4);
+    const float m_q = aqr[R];
+    const float Zt = aqr[R + 1] - zs;                      // Z_hat_R / exp(m_q)
     if (Zt > 0.f) {
       logZR = m_q + logf(Zt);
       Mx = fmaxf(m_E, logZR);
       const float cE = nE > 0 ? expf(m_E - Mx) : 0.f, cR = expf(logZR - Mx);
       if (tid < D) {
-        yR = (red[tid] - zv) / Zt;
+        yR = (aqr[R + 4 + tid] - zv) / Zt;
         y = (cE * nu_E + cR * yR) / (cE * Z_E + cR);
       }
     } else if (tid < D) {

@@ -391,31 +391,81 @@ constexpr int kCompThreads = 256;
 constexpr int kCompPerWarp = kCompactChunk / (kCompThreads / 32);   // 512 scores per warp
 constexpr int kCompIters = kCompPerWarp / 32;                        // 16
 
-// Query-side log-features a_q = W_q q + b_q - gamma_q |q|^2 (Sec. 4.1), kept as
-// exp(a_q - m_q) and m_q so that tiny features cannot underflow the merge.
-__device__ void phi_q_job(const Problem& p, int row, int hq) {
+// Query-side work that does not depend on the selection (Sec. 4.1, Sec. 4.3): the
+// log-features a_q = W_q q + b_q - gamma_q |q|^2, kept as w = exp(a_q - m_q) and m_q so
+// that tiny features cannot underflow the merge, and the unsubtracted residual terms
+// S_M w (d values) and w . u_M.  Row layout of p.aq: [0, r) w, [r] m_q, [r+1] w . u_M,
+// [r+4, r+4+d) S_M w.
+__device__ void phi_q_job(const Problem& p, int row, int hq, int b) {
+  __shared__ float s_q[128];
   __shared__ float s_a[128];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int D = p.head_dim, r = p.n_feat;
-  float* aq = p.aq + (size_t)row * (r + 4);
+  float* aq = p.aq + (size_t)row * (r + D + 4);
   const __nv_bfloat16* qp = p.q + (size_t)row * D;
   const float* W = p.w_q + (size_t)hq * r * D;
+  for (int c = tid; c < D; c += kCompThreads) s_q[c] = __bfloat162float(qp[c]);
+  __syncthreads();
   float qn = 0.f;
-  for (int c = lane; c < D; c += 32) { float x = __bfloat162float(qp[c]); qn = fmaf(x, x, qn); }
+  for (int c = lane; c < D; c += 32) qn = fmaf(s_q[c], s_q[c], qn);
   qn = warp_sum(qn);
-  for (int j = warp; j < r; j += kCompThreads / 32) {
-    float a = 0.f;
-    for (int c = lane; c < D; c += 32) a = fmaf(W[(size_t)j * D + c], __bfloat162float(qp[c]), a);
-    a = warp_sum(a);
-    if (lane == 0) s_a[j] = a + p.b_q[(size_t)hq * r + j] - p.gamma_q * qn;
+  // each warp owns r/8 feature rows: every lane loads its float4 of every row first (all
+  // loads in flight), then the dot products are reduced across the warp
+  constexpr int NW = kCompThreads / 32;
+  constexpr int MAXR = 128 / NW;                      // rows per warp at r = 128
+  const int rows_w = r / NW;
+  float part[MAXR];
+  const bool active = lane * 4 < D;
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    part[i] = 0.f;
+    if (i < rows_w && active) {
+      const float4 w4 = __ldg(reinterpret_cast<const float4*>(W + (size_t)(warp * rows_w + i) * D + lane * 4));
+      part[i] = w4.x * s_q[lane * 4] + w4.y * s_q[lane * 4 + 1] + w4.z * s_q[lane * 4 + 2] + w4.w * s_q[lane * 4 + 3];
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    const float a = warp_sum(part[i]);
+    if (i < rows_w && lane == 0) {
+      const int j = warp * rows_w + i;
+      s_a[j] = a + p.b_q[(size_t)hq * r + j] - p.gamma_q * qn;
+    }
   }
   __syncthreads();
   if (tid < 32) {
     float m = -INFINITY;
     for (int j = tid; j < r; j += 32) m = fmaxf(m, s_a[j]);
     m = warp_max(m);
-    for (int j = tid; j < r; j += 32) aq[j] = expf(s_a[j] - m);
+    for (int j = tid; j < r; j += 32) { const float w = expf(s_a[j] - m); s_a[j] = w; aq[j] = w; }
     if (tid == 0) aq[r] = m;
+  }
+  __syncthreads();
+  // S_M w: one warp per row of S (r floats = up to 32 lanes x float4), rows_d rows per warp
+  const int kvh = hq / p.group;
+  const float* Sg = p.S + ((size_t)b * p.n_kv_heads + kvh) * D * r;
+  const float* ug = p.u + ((size_t)b * p.n_kv_heads + kvh) * r;
+  const int rows_d = D / NW;
+  const bool act_r = lane * 4 < r;
+  float sp[MAXR];
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    sp[i] = 0.f;
+    if (i < rows_d && act_r) {
+      const float4 s4 = __ldg(reinterpret_cast<const float4*>(Sg + (size_t)(warp * rows_d + i) * r + lane * 4));
+      sp[i] = s4.x * s_a[lane * 4] + s4.y * s_a[lane * 4 + 1] + s4.z * s_a[lane * 4 + 2] + s4.w * s_a[lane * 4 + 3];
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    const float a = warp_sum(sp[i]);
+    if (i < rows_d && lane == 0) aq[r + 4 + warp * rows_d + i] = a;
+  }
+  if (warp == 0) {
+    float a = 0.f;
+    for (int j = lane; j < r; j += 32) a = fmaf(ug[j], s_a[j], a);
+    a = warp_sum(a);
+    if (lane == 0) aq[r + 1] = a;
   }
 }
 
@@ -453,7 +503,7 @@ __global__ void __launch_bounds__(kCompThreads) compact_kernel(const Problem p, 
   const int row = b * p.n_q_heads + hq;
   if ((int)blockIdx.x >= n_chunk_ctas) {
     // spare CTAs: feature-map work that does not depend on the scores
-    if ((int)blockIdx.x == n_chunk_ctas) phi_q_job(p, row, hq);
+    if ((int)blockIdx.x == n_chunk_ctas) phi_q_job(p, row, hq, b);
     else if (b == 0 && hq % p.group == 0) wk_split_job(p, hq / p.group);
     return;
   }
