@@ -137,13 +137,13 @@ void build_layout(const tkphi_kv_desc* kv, const Shape& sh, WsLayout* L) {
   L->status = o;        o += 256;
   L->unit_counter = o;  o = align_up(o + sizeof(unsigned) * sh.units, 256);
   L->zero_end = o;
-  // about two CTAs per SM over all units, at least 2048 mid tokens per CTA
-  const int64_t total_mid = (int64_t)sh.max_mid > 0 ? (int64_t)sh.max_mid * sh.units : 0;
-  int64_t chunk = (total_mid + 2 * 148 - 1) / (2 * 148);
-  if (chunk < 2048) chunk = 2048;
-  chunk = (chunk + 31) / 32 * 32;
-  L->chunk_len = (int)chunk;
-  L->chunks_per_unit = sh.max_mid > 0 ? (int)((sh.max_mid + chunk - 1) / chunk) : 1;
+  // one CTA per SM over all units, never more chunks than 128-token tiles
+  const int64_t max_tiles = sh.max_mid > 0 ? ((int64_t)sh.max_mid + 127) / 128 : 1;
+  int64_t cpu = n_sm_cached() / sh.units;
+  if (cpu < 1) cpu = 1;
+  if (cpu > max_tiles) cpu = max_tiles;
+  L->chunk_len = 0;
+  L->chunks_per_unit = (int)cpu;
   L->b_partials = o;
   o = align_up(o + sizeof(float) * (size_t)sh.units * L->chunks_per_unit *
                        ((size_t)kv->head_dim * kv->n_feat + kv->n_feat), 256);
@@ -166,19 +166,20 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 3-D view [head][row][dim] of the key cache; box = 64 dims x one scoring tile of one
-// head, stored with the 128-byte swizzle (head_dim 128 takes two boxes per tile).
-tkphi_status make_key_tensor_map(const tkphi_kv_desc* kv, long long total_tokens, CUtensorMap* tm) {
+// 3-D view [head][row][dim] of a K or V cache; box = 64 dims x box_rows rows of one head,
+// stored with the 128-byte swizzle (head_dim 128 takes two boxes per tile).
+tkphi_status make_tensor_map(const tkphi_kv_desc* kv, const void* base, int box_rows, long long total_tokens,
+                             CUtensorMap* tm) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return fail(TKPHI_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
   const cuuint64_t dims[3] = {(cuuint64_t)kv->head_dim, (cuuint64_t)total_tokens, (cuuint64_t)kv->n_kv_heads};
   const cuuint64_t strides[2] = {(cuuint64_t)kv->kv_stride_token * 2, (cuuint64_t)kv->kv_stride_head * 2};
-  const cuuint32_t box[3] = {64, (cuuint32_t)score_tile_keys(kv->head_dim), 1};   // 128-byte rows
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};   // 128-byte rows
   const cuuint32_t estr[3] = {1, 1, 1};
   // a single head (stride 0 would be rejected): give the unused dimension a legal stride
   cuuint64_t st[2] = {strides[0], strides[1]};
   if (kv->n_kv_heads == 1 || st[1] == 0) st[1] = st[0] * (cuuint64_t)total_tokens;
-  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(kv->k), dims, st, box, estr,
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, st, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(TKPHI_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -286,7 +287,7 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
   if (sh.score_tiles > 0) {
     CUtensorMap tm;
-    st = make_key_tensor_map(kv, sh.total_tokens, &tm);
+    st = make_tensor_map(kv, kv->k, score_tile_keys(kv->head_dim), sh.total_tokens, &tm);
     if (st != TKPHI_OK) return st;
     long long grid = sh.score_tiles < n_sm_cached() ? sh.score_tiles : n_sm_cached();
     {
@@ -370,11 +371,17 @@ tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc
   p.unit_counter = reinterpret_cast<unsigned*>(w + L.unit_counter);
   p.partials = reinterpret_cast<float*>(w + L.b_partials);
   p.chunk_len = L.chunk_len; p.chunks_per_unit = L.chunks_per_unit;
+  if (!aligned16(phi->w_k)) return fail(TKPHI_ERR_INVALID_ARG, "w_k must be 16-byte aligned");
+  CUtensorMap tk, tv;
+  st = make_tensor_map(kv, kv->k, 128, sh.total_tokens, &tk);
+  if (st != TKPHI_OK) return st;
+  st = make_tensor_map(kv, kv->v, 128, sh.total_tokens, &tv);
+  if (st != TKPHI_OK) return st;
   cudaError_t e = cudaMemsetAsync(w, 0, L.zero_end, cs);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_BUILD);
-    e = launch_build(p, cs);
+    e = launch_build(p, tk, tv, cs);
   }
   if (e != cudaSuccess) return cuda_fail(e, "build launch");
   return TKPHI_OK;

@@ -1,45 +1,103 @@
 // Prefill summary build (Sec. 4.1, Eq. natural_cache):
 //   S = sum_{i in M} v_i phi_k(k_i)^T  (d_v x d_phi),   u = sum_{i in M} phi_k(k_i),
 //   phi_k(k) = exp(W_k k + b_k - gamma_k |k|^2).
-// CUDA-core fp32 version: each CTA owns a contiguous chunk of the mid-region of one
-// (sequence, KV head) unit, keeps its share of S in registers, and writes one
-// partial; the last CTA of the unit (atomic ticket) adds the partials in chunk order.
+//
+// Both contractions of the build are dense, so both run on the tensor cores
+// (tcgen05.mma, accumulators in tensor memory).  Per tile of 128 mid-region tokens:
+//   GEMM 1   A^T[j][t] = sum_c W_k[j][c] k_t[c]      A operand: W_k (split into bf16
+//            hi + lo, rows = features, zero padded to 128), B operand: the key tile as
+//            TMA lands it.  The fp32 result sits in tensor memory with one feature per
+//            lane and one token per column.
+//   features Phi^T[j][t] = exp2(A^T + b_j - gamma |k_t|^2) (everything pre-scaled by
+//            log2 e).  Eight warps read the accumulator, add u_j += Phi (fp32), split
+//            Phi into bf16 hi + lo (error ~2^-17) and store both back to tensor memory.
+//   GEMM 2   S^T[j][c] += sum_t Phi^T[j][t] v_t[c]   A operand: Phi^T hi, then lo,
+//            straight from tensor memory; B operand: the value tile as TMA lands it
+//            (tokens along K, dims contiguous).  S^T accumulates in tensor memory over
+//            all tiles of the CTA.
+// Warp roles: 0 TMA producer, 1 MMA issuer, 2..9 feature warps, 10..13 key norms.
+// GEMM 1 of tile i+1 is issued before GEMM 2 of tile i, so the tensor pipe works while
+// the feature warps are busy.  Each CTA owns a contiguous range of tiles of one
+// (sequence, KV head) unit and writes one partial; the last CTA of the unit (atomic
+// ticket, no spinning) adds the partials in chunk order.  Every device-side wait is
+// bounded and reports through the status word.
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace tkphi {
 
-constexpr int kBuildThreads = 256;
-constexpr int kBuildTile = 32;      // tokens per inner tile
+constexpr int kBuildThreads = 448;
+constexpr int kBT = 128;                 // tokens per tile
+constexpr int kBuildTmemCols = 512;
+constexpr int kColD1 = 0;                // two GEMM-1 accumulators of 128 columns (Phi hi overwrites them)
+constexpr int kColD2 = 256;              // S^T accumulator, head_dim columns
+constexpr int kColLo = 384;              // Phi lo, 64 columns per buffer
+constexpr float kLog2e = 1.4426950408889634f;
 
-template <int D, int R>
-struct BuildSmem {
-  static constexpr int WT_LD = R + 1;
-  static constexpr size_t wt = 0;                                       // float [D][R+1]
-  static constexpr size_t kf = wt + sizeof(float) * D * WT_LD;           // float [D][tile]
-  static constexpr size_t vf = kf + sizeof(float) * D * kBuildTile;      // float [tile][D]
-  static constexpr size_t ph = vf + sizeof(float) * D * kBuildTile;      // float [tile][R]
-  static constexpr size_t kn = ph + sizeof(float) * R * kBuildTile;      // float [tile]
-  static constexpr size_t total = kn + sizeof(float) * (kBuildTile + 8);
+template <int D>
+struct BuildCfg {
+  static constexpr int BOXES = D / 64;
+  static constexpr int BOX = kBT * 128;                    // bytes of one 64-dim column block of a tile
+  static constexpr int TILE = BOXES * BOX;                 // 32 KB (d = 128) or 16 KB (d = 64)
+  static constexpr int KS = D == 128 ? 2 : 3;              // key ring stages
+  static constexpr int VS = D == 128 ? 2 : 3;              // value ring stages
+  static constexpr size_t whi = 0;
+  static constexpr size_t wlo = whi + TILE;
+  static constexpr size_t kring = wlo + TILE;
+  static constexpr size_t vring = kring + (size_t)KS * TILE;
+  static constexpr size_t small = vring + (size_t)VS * TILE;
+  // small: barriers (<= 32), snorm[2][128], ucomb[2][128], misc
+  static constexpr size_t total = small + 32 * 8 + 4 * (2 * 128 + 2 * 128 + 16);
 };
 
-template <int D, int R>
-__global__ void __launch_bounds__(kBuildThreads) build_kernel(const BuildProblem p) {
-  using L = BuildSmem<D, R>;
-  extern __shared__ __align__(16) unsigned char smem[];
-  float* Wt = reinterpret_cast<float*>(smem + L::wt);
-  float* kf = reinterpret_cast<float*>(smem + L::kf);
-  float* vf = reinterpret_cast<float*>(smem + L::vf);
-  float* ph = reinterpret_cast<float*>(smem + L::ph);
-  float* knorm = reinterpret_cast<float*>(smem + L::kn);
-  __shared__ int s_last;
+__device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
-  constexpr int TD = D / 16, TR = R / 16;          // register tile of S per thread
-  const int tid = threadIdx.x;
+template <int D>
+__global__ void __launch_bounds__(kBuildThreads, 1)
+build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+             const BuildProblem p) {
+  using C = BuildCfg<D>;
+  constexpr int KS = C::KS, VS = C::VS, BOXES = C::BOXES;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* whi = smem + C::whi;
+  unsigned char* wlo = smem + C::wlo;
+  unsigned char* kring = smem + C::kring;
+  unsigned char* vring = smem + C::vring;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::small);
+  uint64_t* k_full = bars;                 // [KS] key tile landed
+  uint64_t* k_empty = k_full + KS;         // [KS] GEMM 1 and the norm warps are done with it
+  uint64_t* v_full = k_empty + KS;         // [VS]
+  uint64_t* v_empty = v_full + VS;         // [VS] GEMM 2 is done with it
+  uint64_t* d1_full = v_empty + VS;        // [2]  GEMM 1 accumulator complete
+  uint64_t* d1_empty = d1_full + 2;        // [2]  GEMM 2 has consumed the features stored over it
+  uint64_t* p_ready = d1_empty + 2;        // [2]  features stored to tensor memory
+  uint64_t* n_ready = p_ready + 2;         // [2]  key norms of the tile in shared memory
+  uint64_t* d2_full = n_ready + 2;         // [1]  last GEMM 2 complete
+  float* snorm = reinterpret_cast<float*>(bars + 32);        // [2][128]  -gamma log2e |k_t|^2, -inf if masked
+  float* ucomb = snorm + 2 * 128;                            // [2][128]
+  int* misc = reinterpret_cast<int*>(ucomb + 2 * 128);
+  volatile int* s_abort = misc;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 1);
+  int* s_last = misc + 2;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.z, kvh = blockIdx.y, chunk = blockIdx.x;
+  const int R = p.n_feat;
   const int unit = b * p.n_kv_heads + kvh;
   const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
   const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
-  const int n_chunks = (n_mid + p.chunk_len - 1) / p.chunk_len;
   float* S_out = p.S + (size_t)unit * D * R;
   float* u_out = p.u + (size_t)unit * R;
   if (n_mid == 0) {
@@ -49,141 +107,278 @@ __global__ void __launch_bounds__(kBuildThreads) build_kernel(const BuildProblem
     }
     return;
   }
+  const int n_tiles = (n_mid + kBT - 1) / kBT;
+  const int n_chunks = n_tiles < p.chunks_per_unit ? n_tiles : p.chunks_per_unit;
   if (chunk >= n_chunks) return;
-  const int m0 = chunk * p.chunk_len;
-  const int m1 = min(n_mid, m0 + p.chunk_len);
+  const int t0 = (int)((long long)n_tiles * chunk / n_chunks);
+  const int t1 = (int)((long long)n_tiles * (chunk + 1) / n_chunks);
+  const int n_my = t1 - t0;                                   // >= 1
+  const int row0 = (int)(cu_b + p.n_sink);                    // cache row of mid token 0
 
-  const float* W = p.w_k + (size_t)kvh * R * D;
-  for (int i = tid; i < R * D; i += kBuildThreads) Wt[(i % D) * L::WT_LD + (i / D)] = W[i];
-
-  const __nv_bfloat16* kbase = p.k + (long long)kvh * p.stride_head + (cu_b + p.n_sink) * p.stride_token;
-  const __nv_bfloat16* vbase = p.v + (long long)kvh * p.stride_head + (cu_b + p.n_sink) * p.stride_token;
-
-  // phase-1 mapping: feature j, token group tg
-  constexpr int NG = kBuildThreads / R, TPG = kBuildTile / NG;
-  const int j = tid % R, tg = tid / R, t0 = tg * TPG;
-  const float bj = p.b_k[(size_t)kvh * R + j];
-  // phase-2 mapping: S rows [TD*ti, +TD), columns [TR*tj, +TR)
-  const int ti = tid / 16, tj = tid % 16;
-  float acc[TD][TR];
+  // ---- set-up: barriers, tensor memory, W_k operand tiles (scaled by log2 e, hi + lo)
+  if (tid == 0) {
+    for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 5); }
+    for (int s = 0; s < VS; ++s) { mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&d1_full[s], 1); mbar_init(&d1_empty[s], 1); mbar_init(&p_ready[s], 8); mbar_init(&n_ready[s], 4);
+    }
+    mbar_init(d2_full, 1);
+    mbar_fence_init();
+    *s_abort = 0;
+  }
+  if (warp == 1) tmem_alloc(s_tmem, kBuildTmemCols);
+  {
+    const float* W = p.w_k + (size_t)kvh * R * D;
+    constexpr int CPR = D / 8;
+    for (int i = tid; i < 128 * CPR; i += kBuildThreads) {
+      const int row = i / CPR, c = i % CPR;
+      unsigned hw[4] = {0, 0, 0, 0}, lw[4] = {0, 0, 0, 0};
+      if (row < R) {
+        const float4 w0 = *reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8);
+        const float4 w1 = *reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8 + 4);
+        const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
-  for (int a = 0; a < TD; ++a)
-#pragma unroll
-    for (int c = 0; c < TR; ++c) acc[a][c] = 0.f;
-  float uacc = 0.f;
-
-  constexpr int CPR = D / 8;
-  for (int base = m0; base < m1; base += kBuildTile) {
-    __syncthreads();
-    for (int i = tid; i < kBuildTile * CPR; i += kBuildThreads) {
-      const int t = i / CPR, c = i % CPR;
-      uint4 kraw = make_uint4(0, 0, 0, 0), vraw = make_uint4(0, 0, 0, 0);
-      if (base + t < m1) {
-        kraw = *reinterpret_cast<const uint4*>(kbase + (long long)(base + t) * p.stride_token + c * 8);
-        vraw = *reinterpret_cast<const uint4*>(vbase + (long long)(base + t) * p.stride_token + c * 8);
+        for (int e = 0; e < 4; ++e) {
+          const float a0 = w[2 * e] * kLog2e, a1 = w[2 * e + 1] * kLog2e;
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(a0), h1 = __float2bfloat16_rn(a1);
+          const __nv_bfloat16 l0 = __float2bfloat16_rn(a0 - __bfloat162float(h0));
+          const __nv_bfloat16 l1 = __float2bfloat16_rn(a1 - __bfloat162float(h1));
+          hw[e] = (unsigned)__bfloat16_as_ushort(h0) | ((unsigned)__bfloat16_as_ushort(h1) << 16);
+          lw[e] = (unsigned)__bfloat16_as_ushort(l0) | ((unsigned)__bfloat16_as_ushort(l1) << 16);
+        }
       }
-      const unsigned kw[4] = {kraw.x, kraw.y, kraw.z, kraw.w};
-      const unsigned vw[4] = {vraw.x, vraw.y, vraw.z, vraw.w};
+      const uint32_t off = (c >> 3) * C::BOX + swz128(row, c & 7);
+      *reinterpret_cast<uint4*>(whi + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      *reinterpret_cast<uint4*>(wlo + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+    }
+  }
+  fence_proxy_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *s_tmem;
+
+  if (warp == 0) {
+    // ================================================================ TMA producer
+    if (lane == 0) {
+      bool ok = true;
+      for (int it = 0; it < n_my && ok; ++it) {
+        const int row = row0 + (t0 + it) * kBT;
+        const int ks = it % KS, vs = it % VS;
+        ok = mbar_wait(&k_empty[ks], ((uint32_t)(it / KS) & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+        mbar_expect_tx(&k_full[ks], C::TILE);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        kf[(c * 8 + 2 * e) * kBuildTile + t] = bf16_lo(kw[e]);
-        kf[(c * 8 + 2 * e + 1) * kBuildTile + t] = bf16_hi(kw[e]);
-        vf[t * D + c * 8 + 2 * e] = bf16_lo(vw[e]);
-        vf[t * D + c * 8 + 2 * e + 1] = bf16_hi(vw[e]);
+        for (int x = 0; x < BOXES; ++x)
+          tma_load_3d(kring + ks * C::TILE + x * C::BOX, &tmap_k, &k_full[ks], x * 64, row, kvh);
+        ok = mbar_wait(&v_empty[vs], ((uint32_t)(it / VS) & 1u) ^ 1u, s_abort);
+        if (!ok) {
+          // the key copy just issued must land before shared memory is released
+          for (uint32_t w = 0; w < kWaitPolls; ++w) {
+            if (mbar_try_wait(&k_full[ks], (uint32_t)(it / KS) & 1u)) break;
+            __nanosleep(64);
+          }
+          break;
+        }
+        mbar_expect_tx(&v_full[vs], C::TILE);
+#pragma unroll
+        for (int x = 0; x < BOXES; ++x)
+          tma_load_3d(vring + vs * C::TILE + x * C::BOX, &tmap_v, &v_full[vs], x * 64, row, kvh);
       }
     }
-    __syncthreads();
-    if (tid < kBuildTile) {
+  } else if (warp == 1) {
+    // ================================================================ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc1 = umma_idesc_bf16(128, kBT, 0, 0);
+      constexpr uint32_t idesc2 = umma_idesc_bf16(128, D, 0, 1);
+      const uint64_t whi_d = umma_smem_desc(smem_u32(whi), 16, 1024);
+      const uint64_t wlo_d = umma_smem_desc(smem_u32(wlo), 16, 1024);
+      const uint64_t k_d = umma_smem_desc(smem_u32(kring), 16, 1024);
+      // value tile as an MN-major operand: 64-dim column blocks BOX bytes apart, groups of
+      // eight token rows 1024 bytes apart
+      const uint64_t v_d = umma_smem_desc(smem_u32(vring), C::BOX, 1024);
+      bool ok = true;
+      auto gemm2 = [&](int j) {
+        const int buf = j & 1, vs = j % VS;
+        ok = mbar_wait(&p_ready[buf], (uint32_t)(j >> 1) & 1u, s_abort) &&
+             mbar_wait(&v_full[vs], (uint32_t)(j / VS) & 1u, s_abort);
+        if (!ok) return;
+        tc_fence_after_sync();
+        const uint64_t vd = v_d + (uint64_t)((vs * C::TILE) >> 4);
+#pragma unroll
+        for (int kk = 0; kk < kBT / 16; ++kk) {
+          // tokens 16 kk .. 16 kk + 15: eight packed columns of Phi hi, then of Phi lo
+          const uint32_t hi_col = kColD1 + buf * 128 + (kk >> 2) * 64 + ((kk >> 1) & 1) * 16 + (kk & 1) * 8;
+          const uint32_t lo_col = kColLo + buf * 64 + (kk >> 2) * 32 + ((kk >> 1) & 1) * 16 + (kk & 1) * 8;
+          const uint64_t bd = vd + (uint64_t)((kk * 16 * 128) >> 4);
+          umma_ts(tmem_base + kColD2, tmem_base + hi_col, bd, idesc2, (j > 0 || kk > 0) ? 1u : 0u);
+          umma_ts(tmem_base + kColD2, tmem_base + lo_col, bd, idesc2, 1u);
+        }
+        tc_commit(&v_empty[vs]);
+        tc_commit(&d1_empty[buf]);
+      };
+      for (int it = 0; it < n_my && ok; ++it) {
+        const int buf = it & 1, ks = it % KS;
+        ok = mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort) &&
+             mbar_wait(&d1_empty[buf], ((uint32_t)(it >> 1) & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t kd = k_d + (uint64_t)((ks * C::TILE) >> 4);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint64_t wd = half == 0 ? whi_d : wlo_d;
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            const uint64_t off = (uint64_t)(((k >> 2) * C::BOX + (k & 3) * 32) >> 4);
+            umma_ss(tmem_base + kColD1 + buf * 128, wd + off, kd + off, idesc1, (half | k) ? 1u : 0u);
+          }
+        }
+        tc_commit(&d1_full[buf]);
+        tc_commit(&k_empty[ks]);
+        if (it > 0) gemm2(it - 1);
+      }
+      if (ok) gemm2(n_my - 1);
+      if (ok) tc_commit(d2_full);
+    }
+  } else if (warp < 10) {
+    // ================================================================ feature warps
+    const int quad = warp & 3;                     // tensor-memory lane quadrant
+    const int h = (warp - 2) >> 2;                 // which 64 tokens of the tile
+    const int j = quad * 32 + lane;                // feature
+    const float bj = j < R ? p.b_k[(size_t)kvh * R + j] * kLog2e : 0.f;
+    float u_acc = 0.f;                             // sum of feature j over this thread's tokens
+    bool ok = true;
+    for (int it = 0; it < n_my && ok; ++it) {
+      const int buf = it & 1;
+      const uint32_t ph = (uint32_t)(it >> 1) & 1u;
+      ok = mbar_wait(&d1_full[buf], ph, s_abort) && mbar_wait(&n_ready[buf], ph, s_abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const float* sn = snorm + buf * 128 + h * 64;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        float v[32];
+        tmem_ld_x32(tmem_addr(tmem_base, quad * 32, kColD1 + buf * 128 + h * 64 + c * 32), v);
+        tc_wait_ld();
+        uint32_t hi[16], lo[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float f0 = ex2_approx(v[2 * e] + bj + sn[c * 32 + 2 * e]);
+          const float f1 = ex2_approx(v[2 * e + 1] + bj + sn[c * 32 + 2 * e + 1]);
+          u_acc += f0;
+          u_acc += f1;
+          const __nv_bfloat162 hp = __floats2bfloat162_rn(f0, f1);          // .x (low half) = even token
+          const __nv_bfloat162 lp =
+              __floats2bfloat162_rn(f0 - __bfloat162float(hp.x), f1 - __bfloat162float(hp.y));
+          hi[e] = *reinterpret_cast<const uint32_t*>(&hp);
+          lo[e] = *reinterpret_cast<const uint32_t*>(&lp);
+        }
+        // hi goes over columns of this thread's own region that it has already read
+        tmem_st_x16(tmem_addr(tmem_base, quad * 32, kColD1 + buf * 128 + h * 64 + c * 16), hi);
+        tmem_st_x16(tmem_addr(tmem_base, quad * 32, kColLo + buf * 64 + h * 32 + c * 16), lo);
+      }
+      tc_wait_st();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_ready[buf]);
+    }
+    // ---- S^T of this CTA's tiles -> partial (thread = feature, h = half of the dims)
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(d2_full, 0, s_abort));
+    if (ok) {
+      tc_fence_after_sync();
+      float* part = p.partials + ((size_t)unit * p.chunks_per_unit + chunk) * ((size_t)D * R + R);
+      constexpr int HALF = D / 2;
+#pragma unroll
+      for (int c = 0; c < HALF / 32; ++c) {
+        float v[32];
+        tmem_ld_x32(tmem_addr(tmem_base, quad * 32, kColD2 + h * HALF + c * 32), v);
+        tc_wait_ld();
+        if (j < R) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) part[(size_t)(h * HALF + c * 32 + e) * R + j] = v[e];
+        }
+      }
+      ucomb[h * 128 + j] = u_acc;
+    }
+  } else {
+    // ================================================================ key norms and masking
+    const int t = (warp - 10) * 32 + lane;         // token of the tile
+    const float g2 = p.gamma_k * kLog2e;
+    bool ok = true;
+    for (int it = 0; it < n_my && ok; ++it) {
+      const int buf = it & 1, ks = it % KS;
+      ok = mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort) &&
+           mbar_wait(&d1_empty[buf], ((uint32_t)(it >> 1) & 1u) ^ 1u, s_abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const unsigned char* tile = kring + ks * C::TILE;
       float kn = 0.f;
-      for (int c = 0; c < D; ++c) { const float x = kf[c * kBuildTile + tid]; kn = fmaf(x, x, kn); }
-      knorm[tid] = kn;
-    }
-    // phi_k for the tile
-    float a[TPG];
 #pragma unroll
-    for (int t = 0; t < TPG; ++t) a[t] = 0.f;
-    for (int c = 0; c < D; ++c) {
-      const float w = Wt[c * L::WT_LD + j];
-      const float4* kp = reinterpret_cast<const float4*>(kf + c * kBuildTile + t0);
+      for (int c = 0; c < D / 8; ++c) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(tile + (c >> 3) * C::BOX + swz128(t, c & 7));
+        const unsigned w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-      for (int t4 = 0; t4 < TPG / 4; ++t4) {
-        const float4 kv = kp[t4];
-        a[4 * t4 + 0] = fmaf(w, kv.x, a[4 * t4 + 0]);
-        a[4 * t4 + 1] = fmaf(w, kv.y, a[4 * t4 + 1]);
-        a[4 * t4 + 2] = fmaf(w, kv.z, a[4 * t4 + 2]);
-        a[4 * t4 + 3] = fmaf(w, kv.w, a[4 * t4 + 3]);
+        for (int e = 0; e < 4; ++e) {
+          const float x0 = bf16_lo(w[e]), x1 = bf16_hi(w[e]);
+          kn = fmaf(x0, x0, kn);
+          kn = fmaf(x1, x1, kn);
+        }
       }
-    }
-    __syncthreads();                                   // knorm visible
-#pragma unroll
-    for (int t = 0; t < TPG; ++t) {
-      const float f = (base + t0 + t < m1) ? expf(a[t] + bj - p.gamma_k * knorm[t0 + t]) : 0.f;
-      ph[(t0 + t) * R + j] = f;
-    }
-    __syncthreads();
-    // S += V^T Phi, u += column sums of Phi
-    for (int t = 0; t < kBuildTile; ++t) {
-      float vv[TD], pp[TR];
-#pragma unroll
-      for (int x = 0; x < TD; x += 4) {
-        const float4 q4 = *reinterpret_cast<const float4*>(vf + t * D + TD * ti + x);
-        vv[x] = q4.x; vv[x + 1] = q4.y; vv[x + 2] = q4.z; vv[x + 3] = q4.w;
-      }
-#pragma unroll
-      for (int x = 0; x < TR; x += 4) {
-        const float4 q4 = *reinterpret_cast<const float4*>(ph + t * R + TR * tj + x);
-        pp[x] = q4.x; pp[x + 1] = q4.y; pp[x + 2] = q4.z; pp[x + 3] = q4.w;
-      }
-#pragma unroll
-      for (int x = 0; x < TD; ++x)
-#pragma unroll
-        for (int y = 0; y < TR; ++y) acc[x][y] = fmaf(vv[x], pp[y], acc[x][y]);
-    }
-    if (tid < R) {
-      for (int t = 0; t < kBuildTile; ++t) uacc += ph[t * R + tid];
+      const bool valid = (t0 + it) * kBT + t < n_mid;
+      snorm[buf * 128 + t] = valid ? -g2 * kn : -INFINITY;   // exp2(-inf) = 0 removes rows outside the mid-region
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&n_ready[buf]); mbar_arrive(&k_empty[ks]); }
     }
   }
 
-  // ---- partial of this chunk
-  float* part = p.partials + ((size_t)unit * p.chunks_per_unit + chunk) * (D * R + R);
-#pragma unroll
-  for (int x = 0; x < TD; ++x)
-#pragma unroll
-    for (int y = 0; y < TR; ++y) part[(TD * ti + x) * R + TR * tj + y] = acc[x][y];
-  if (tid < R) part[D * R + tid] = uacc;
+  // ---- teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kBuildTmemCols);
+  }
+  if (*s_abort) {
+    if (tid == 0) atomicExch(p.status, kStatusTimeout);
+    return;
+  }
+  float* part = p.partials + ((size_t)unit * p.chunks_per_unit + chunk) * ((size_t)D * R + R);
+  if (tid < R) part[(size_t)D * R + tid] = ucomb[tid] + ucomb[128 + tid];
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&p.unit_counter[unit], 1u) == (unsigned)(n_chunks - 1));
+  if (tid == 0) *s_last = (atomicAdd(&p.unit_counter[unit], 1u) == (unsigned)(n_chunks - 1));
   __syncthreads();
-  if (!s_last) return;
+  if (!*s_last) return;
   __threadfence();
-  const float* parts = p.partials + (size_t)unit * p.chunks_per_unit * (D * R + R);
+  // last CTA of the unit: add the chunk partials in chunk order
+  const float* parts = p.partials + (size_t)unit * p.chunks_per_unit * ((size_t)D * R + R);
   for (int i = tid; i < D * R + R; i += kBuildThreads) {
     float s = 0.f;
-    for (int c = 0; c < n_chunks; ++c) s += __ldcg(parts + (size_t)c * (D * R + R) + i);
+#pragma unroll 4
+    for (int c = 0; c < n_chunks; ++c) s += __ldcg(parts + (size_t)c * ((size_t)D * R + R) + i);
     if (i < D * R) S_out[i] = s; else u_out[i - D * R] = s;
   }
 }
 
-template <int D, int R>
-static cudaError_t launch_build_t(const BuildProblem& p, cudaStream_t st) {
+template <int D>
+static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, const CUtensorMap& tv,
+                                  cudaStream_t st) {
   static bool configured = false;
-  const size_t smem = BuildSmem<D, R>::total;
+  const size_t smem = BuildCfg<D>::total;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(build_kernel<D, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(build_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   dim3 grid(p.chunks_per_unit, p.n_kv_heads, p.batch);
-  build_kernel<D, R><<<grid, kBuildThreads, smem, st>>>(p);
+  build_kernel<D><<<grid, kBuildThreads, smem, st>>>(tk, tv, p);
   return cudaGetLastError();
 }
 
-cudaError_t launch_build(const BuildProblem& p, cudaStream_t st) {
-  if (p.head_dim == 64 && p.n_feat == 64) return launch_build_t<64, 64>(p, st);
-  if (p.head_dim == 64 && p.n_feat == 128) return launch_build_t<64, 128>(p, st);
-  if (p.head_dim == 128 && p.n_feat == 64) return launch_build_t<128, 64>(p, st);
-  if (p.head_dim == 128 && p.n_feat == 128) return launch_build_t<128, 128>(p, st);
+cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tk, const CUtensorMap& tv, cudaStream_t st) {
+  if (p.head_dim == 64) return launch_build_t<64>(p, tk, tv, st);
+  if (p.head_dim == 128) return launch_build_t<128>(p, tk, tv, st);
   return cudaErrorInvalidValue;
 }
 

@@ -71,7 +71,7 @@ struct BuildProblem {
   int* status;
   unsigned* unit_counter;          // [batch*n_kv_heads]
   float* partials;                 // [units][chunks_per_unit][d*r + r]
-  int chunk_len;                   // mid tokens per CTA
+  int chunk_len;                   // unused
   int chunks_per_unit;             // upper bound over sequences
 };
 
@@ -167,6 +167,6 @@ cudaError_t launch_hist(const Problem& p, int max_mid, cudaStream_t stream);
 cudaError_t launch_compact(const Problem& p, int max_mid, cudaStream_t stream);
 cudaError_t launch_finalize_select(const Problem& p, cudaStream_t stream);
 cudaError_t launch_exact_residual(const Problem& p, cudaStream_t stream);
-cudaError_t launch_build(const BuildProblem& p, cudaStream_t stream);
+cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, cudaStream_t stream);
 
 }  // namespace tkphi
