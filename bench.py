@@ -35,12 +35,18 @@ L2_BYTES = 126e6
 
 
 def _peaks():
+    """(HBM GB/s, bf16 TFLOP/s burst, bf16 TFLOP/s sustained, "measured" | "fallback")."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+    return 6650.0, 1590.0, 1400.0, "fallback"
+
+
+# DRAM bytes per launch of the scoring kernel from the committed ncu capture of this kernel
+# (profiles/); None once the kernel has changed since the capture.
+SCORE_KERNEL_NCU_TRAFFIC_BYTES = None
 
 
 # --------------------------------------------------------------------------- clocks
@@ -227,7 +233,7 @@ def run_ours(args, rank, world, device):
         ms, e2e_ms = float(t[0]), float(t[1])
 
     ab = algorithmic_bytes(cfg, N, tmax, n_layers)
-    peak, peak_kind = _peaks()
+    peak, tf_burst, tf_sust, peak_kind = _peaks()
     out = {
         "metric": "Top-K+phi decode-step latency (us), 128K ctx",
         "value": ms * 1e3, "unit": "us/step", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -243,10 +249,10 @@ def run_ours(args, rank, world, device):
         "hbm_frac_of_measured_peak": ab["total"] / (ms * 1e-3) / 1e9 / peak,
         "algorithmic_bytes_per_step": ab["total"],
         "steps_per_s_all_gpus": world * 1e3 / ms,
-        "gpu_launches": args.steps * n_layers * 4,
+        "gpu_launches": args.steps * n_layers * 5,
         "e2e": {"value": e2e_ms * 1e3, "unit": "us/step", "h2d_bytes_per_step": q_stage.numel() * 2,
                 "d2h_bytes_per_step": y_host.numel() * 4},
-        "build": {"ms_all_layers": build_ms, "kv_bytes": 2 * n_layers * Hkv * (N - cfg.n_sink - cfg.n_tail) * d * 2 * B},
+        "build": build_info(build_ms, n_layers, B, Hkv, N - cfg.n_sink - cfg.n_tail, d, r, peak, tf_burst, tf_sust),
         "clocks": clocks,
         "gen_s": t_gen,
     }
@@ -254,10 +260,24 @@ def run_ours(args, rank, world, device):
         dom = kt["score"]
         a = ab["key_stream_per_layer"] / (dom["avg_ms"] * 1e-3) / 1e9
         out["roofline"] = {"bound": "hbm", "kernel": "score_kernel", "achieved": a, "peak": peak,
-                           "unit": "GB/s", "frac": a / peak, "traffic": None, "peak_kind": peak_kind,
+                           "unit": "GB/s", "frac": a / peak, "traffic": SCORE_KERNEL_NCU_TRAFFIC_BYTES,
+                           "peak_kind": peak_kind, "algorithmic_bytes_per_launch": ab["key_stream_per_layer"],
                            "avg_launch_us": dom["avg_ms"] * 1e3}
         out["kernels_us_per_launch"] = {k: v["avg_ms"] * 1e3 for k, v in kt.items()}
     return out, (cfg, layers, phis, Ss, us, topk)
+
+
+def build_info(build_ms, n_layers, B, Hkv, n_mid, d, r, hbm_peak, tf_burst, tf_sust):
+    """Prefill summary build, timed separately: K and V of the mid-region are read once;
+    the two contractions cost 2 * (2 n d r) flop per KV head, issued twice each (bf16 hi + lo)."""
+    kv_bytes = 2 * n_layers * B * Hkv * n_mid * d * 2
+    flops_alg = 4.0 * n_layers * B * Hkv * n_mid * d * r
+    t = build_ms * 1e-3
+    return {"ms_all_layers": build_ms, "kv_bytes": kv_bytes, "achieved_gbs": kv_bytes / t / 1e9,
+            "hbm_frac_of_measured_peak": kv_bytes / t / 1e9 / hbm_peak,
+            "algorithmic_tflops": flops_alg / t / 1e12, "issued_tflops_bf16": 2 * flops_alg / t / 1e12,
+            "issued_frac_of_bf16_burst_peak": 2 * flops_alg / t / 1e12 / tf_burst,
+            "issued_frac_of_bf16_sustained_peak": 2 * flops_alg / t / 1e12 / tf_sust}
 
 
 # --------------------------------------------------------------------------- oracle legs
