@@ -279,28 +279,31 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   // idx_out uses the caller's topk_max as its row length; the internal list uses p.topk_max
   if (topk_max == 0) p.idx_out = nullptr;
 
+  p.zero_bytes = L.zero_end;
   cudaError_t e;
-  {
-    ScopedSpan sp(cs, TKPHI_KERNEL_MEMSET);
-    e = cudaMemsetAsync(w, 0, L.zero_end, cs);
-  }
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
+  // The scoring kernel also clears the workspace counters; without keys to score a plain
+  // memset does.  The histogram and compaction kernels carry the query-side feature work
+  // on spare CTAs, so they are launched (possibly with no score chunks) whenever there are
+  // feature maps.
   if (sh.score_tiles > 0) {
     CUtensorMap tm;
     st = make_tensor_map(kv, kv->k, score_tile_keys(kv->head_dim), sh.total_tokens, &tm);
     if (st != TKPHI_OK) return st;
-    long long grid = sh.score_tiles < n_sm_cached() ? sh.score_tiles : n_sm_cached();
     {
       ScopedSpan sp(cs, TKPHI_KERNEL_SCORE);
-      e = launch_score(p, tm, (int)grid, cs);
+      e = launch_score(p, tm, n_sm_cached(), cs);
     }
     if (e != cudaSuccess) return cuda_fail(e, "score launch");
-    {
-      ScopedSpan sp(cs, TKPHI_KERNEL_HIST);
-      e = launch_hist(p, sh.max_mid, cs);
-    }
-    if (e != cudaSuccess) return cuda_fail(e, "hist launch");
+  } else {
+    ScopedSpan sp(cs, TKPHI_KERNEL_MEMSET);
+    e = cudaMemsetAsync(w, 0, L.zero_end, cs);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
   }
+  {
+    ScopedSpan sp(cs, TKPHI_KERNEL_HIST);
+    e = launch_hist(p, sh.score_tiles > 0 ? sh.max_mid : 0, cs);
+  }
+  if (e != cudaSuccess) return cuda_fail(e, "hist launch");
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_COMPACT);
     e = launch_compact(p, sh.score_tiles > 0 ? sh.max_mid : 0, cs);

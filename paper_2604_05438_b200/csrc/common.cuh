@@ -15,7 +15,7 @@ constexpr int kHistBins = 1 << kHistBits;     // bins of the fused first-pass hi
 constexpr int kLowBits = 32 - kHistBits;      // bits refined inside the threshold bin
 constexpr int kMaxBatch = 1024;               // sequences per call
 constexpr int kSlice = 128;                   // exact-support tokens per CTA of the exact/residual kernel (= MMA M)
-constexpr int kCompactChunk = 4096;           // scores per CTA of the compaction kernel
+constexpr int kCompactChunk = 16384;          // scores per CTA of the compaction kernel
 constexpr int kMaxChunks = 2048;              // compaction chunks per sequence the selection kernel can index
 
 // Device status word values (first word of the workspace).
@@ -42,7 +42,8 @@ struct Problem {
   unsigned flags;
   int with_phi;                    // 0: selection-only, 1: Top-K+phi
   // workspace pieces (device pointers)
-  int* status;
+  int* status;                     // first word of the workspace
+  size_t zero_bytes;               // head of the workspace that must be zero before the selection kernels
   unsigned* unit_counter;          // [batch*n_q_heads] histogram-chunk tickets
   unsigned* row_counter;           // [batch*n_q_heads]
   int4* rowinfo;                   // [rows]: x = threshold bin, y = count above, z = count in bin

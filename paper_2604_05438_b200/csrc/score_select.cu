@@ -10,15 +10,15 @@
 //                          from shared memory and the group's queries (zero padded) as the
 //                          other, so the dot products cost no issue slots of the CUDA cores;
 //                          one warp reads the fp32 accumulators back from tensor memory and
-//                          writes the score rows.
+//                          writes the score rows.  The CTAs also clear the workspace counters.
 //   hist_kernel            one pass over the (L2-resident) scores: 4096-bin histogram of the
 //                          leading 12 bits of the order-preserving score key per query head;
-//                          the last CTA of a head turns it into a threshold bin.
+//                          the last CTA of a head turns it into a threshold bin.  A spare CTA
+//                          per head evaluates the query's log-features and splits W_k.
 //   compact_kernel         one pass over the (L2-resident) scores: a bitmap of positions above
 //                          the threshold bin and, per 4096-score chunk, the ordered list of
-//                          positions inside it.  Spare CTAs evaluate the query-side
-//                          log-features and split W_k into bf16 operand tiles for the
-//                          retrieved-key feature recompute.
+//                          positions inside it.  A spare CTA per head contracts the summaries
+//                          with the query features (the unsubtracted residual terms).
 //   finalize_select_kernel one CTA per query head: radix-refines the remaining 20 key bits
 //                          among the candidates (in shared memory), admits exact ties in index
 //                          order, and expands the final bitmap into the ascending index list.
@@ -74,6 +74,134 @@ __device__ __forceinline__ void cursor_next(TileCursor& c, const int* pre, int b
   } while (c.nt == 0);
 }
 
+// ------------------------------------------------------------------ query-side feature work
+// Work that depends only on the call's inputs is done by spare CTAs of the two selection
+// kernels that stream the (L2-resident) scores, where it is off the critical path and the
+// memory system is not saturated: stage 1 (log-features of the query) with the histogram
+// pass, stage 2 (unsubtracted residual terms) with the compaction pass.
+//
+// Query-side quantities (Sec. 4.1, Sec. 4.3): a_q = W_q q + b_q - gamma_q |q|^2, kept as
+// w = exp(a_q - m_q) and m_q so that tiny features cannot underflow the merge, and the
+// unsubtracted residual terms S_M w (d values) and w . u_M.  Row layout of p.aq:
+// [0, r) w, [r] m_q, [r+1] w . u_M, [r+4, r+4+d) S_M w.
+
+// Stage 1, by all NT threads of a CTA: w and m_q of query row `row`.
+template <int NT>
+__device__ void phi_q_stage1(const Problem& p, int row) {
+  __shared__ float s_q[128];
+  __shared__ float s_a[128];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int D = p.head_dim, r = p.n_feat;
+  const int hq = row % p.n_q_heads;
+  float* aq = p.aq + (size_t)row * (r + D + 4);
+  const __nv_bfloat16* qp = p.q + (size_t)row * D;
+  const float* W = p.w_q + (size_t)hq * r * D;
+  for (int c = tid; c < D; c += NT) s_q[c] = __bfloat162float(qp[c]);
+  // each warp owns r/NW feature rows: every lane loads its float4 of every row first (all
+  // loads in flight), then the dot products are reduced across the warp
+  constexpr int NW = NT / 32;
+  constexpr int MAXR = 128 / NW;                      // rows per warp at r = 128
+  const int rows_w = r / NW;
+  float4 w4[MAXR];
+  float bq[MAXR];
+  const bool active = lane * 4 < D;
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    w4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    bq[i] = 0.f;
+    if (i < rows_w) {
+      if (active) w4[i] = __ldg(reinterpret_cast<const float4*>(W + (size_t)(warp * rows_w + i) * D + lane * 4));
+      bq[i] = __ldg(p.b_q + (size_t)hq * r + warp * rows_w + i);
+    }
+  }
+  __syncthreads();
+  float qn = 0.f;
+  for (int c = lane; c < D; c += 32) qn = fmaf(s_q[c], s_q[c], qn);
+  qn = warp_sum(qn);
+  const float q0 = active ? s_q[lane * 4] : 0.f, q1 = active ? s_q[lane * 4 + 1] : 0.f;
+  const float q2 = active ? s_q[lane * 4 + 2] : 0.f, q3 = active ? s_q[lane * 4 + 3] : 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    const float a = warp_sum(w4[i].x * q0 + w4[i].y * q1 + w4[i].z * q2 + w4[i].w * q3);
+    if (i < rows_w && lane == 0) s_a[warp * rows_w + i] = a + bq[i] - p.gamma_q * qn;
+  }
+  __syncthreads();
+  float m = -INFINITY;
+  for (int j = lane; j < r; j += 32) m = fmaxf(m, s_a[j]);
+  m = warp_max(m);                                    // every warp computes the same maximum
+  if (tid < r) aq[tid] = expf(s_a[tid] - m);
+  if (tid == 0) aq[r] = m;
+}
+
+// Stage 2, by all NT threads of a CTA of a later kernel: S_M w and w . u_M of query row `row`.
+template <int NT>
+__device__ void phi_q_stage2(const Problem& p, int row) {
+  __shared__ float s_w[128];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int D = p.head_dim, r = p.n_feat;
+  const int b = row / p.n_q_heads, hq = row % p.n_q_heads, kvh = hq / p.group;
+  float* aq = p.aq + (size_t)row * (r + D + 4);
+  const float* Sg = p.S + ((size_t)b * p.n_kv_heads + kvh) * D * r;
+  const float* ug = p.u + ((size_t)b * p.n_kv_heads + kvh) * r;
+  constexpr int NW = NT / 32;
+  constexpr int MAXR = 128 / NW;
+  const int rows_d = D / NW;
+  const bool act_r = lane * 4 < r;
+  float4 s4[MAXR];
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    s4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < rows_d && act_r)
+      s4[i] = __ldg(reinterpret_cast<const float4*>(Sg + (size_t)(warp * rows_d + i) * r + lane * 4));
+  }
+  if (tid < r) s_w[tid] = __ldcg(aq + tid);            // written by stage 1 in an earlier kernel
+  __syncthreads();
+  const float w0 = act_r ? s_w[lane * 4] : 0.f, w1 = act_r ? s_w[lane * 4 + 1] : 0.f;
+  const float w2 = act_r ? s_w[lane * 4 + 2] : 0.f, w3 = act_r ? s_w[lane * 4 + 3] : 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXR; ++i) {
+    const float a = warp_sum(s4[i].x * w0 + s4[i].y * w1 + s4[i].z * w2 + s4[i].w * w3);
+    if (i < rows_d && lane == 0) aq[r + 4 + warp * rows_d + i] = a;
+  }
+  if (warp == 0) {
+    float a = 0.f;
+    for (int j = lane; j < r; j += 32) a = fmaf(__ldg(ug + j), s_w[j], a);
+    a = warp_sum(a);
+    if (lane == 0) aq[r + 1] = a;
+  }
+}
+
+// W_k of one KV head (fp32 [r][d]) -> two bf16 images, hi = bf16(W) and lo = bf16(W - hi),
+// each laid out as the K-major, 128B-swizzled B operand of the feature recompute MMA:
+// [d/64 column blocks][r rows][128 bytes].  By all NT threads of a CTA.
+template <int NT>
+__device__ void wk_split_job(const Problem& p, int kvh) {
+  const int D = p.head_dim, r = p.n_feat;
+  const float* W = p.w_k + (size_t)kvh * r * D;
+  unsigned char* hi = reinterpret_cast<unsigned char*>(p.wk_img + (size_t)kvh * 2 * r * D);
+  unsigned char* lo = hi + (size_t)r * D * 2;
+  const int cpr = D / 8;
+#pragma unroll 4
+  for (int i = threadIdx.x; i < r * cpr; i += NT) {
+    const int row = i / cpr, c = i % cpr;
+    const float4 w0 = __ldg(reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8));
+    const float4 w1 = __ldg(reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8 + 4));
+    const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+    unsigned hw[4], lw[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(w[2 * e]), h1 = __float2bfloat16_rn(w[2 * e + 1]);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(w[2 * e] - __bfloat162float(h0));
+      const __nv_bfloat16 l1 = __float2bfloat16_rn(w[2 * e + 1] - __bfloat162float(h1));
+      hw[e] = (unsigned)__bfloat16_as_ushort(h0) | ((unsigned)__bfloat16_as_ushort(h1) << 16);
+      lw[e] = (unsigned)__bfloat16_as_ushort(l0) | ((unsigned)__bfloat16_as_ushort(l1) << 16);
+    }
+    const size_t off = (size_t)(c >> 3) * r * 128 + swz128(row, c & 7);
+    *reinterpret_cast<uint4*>(hi + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+    *reinterpret_cast<uint4*>(lo + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+  }
+}
+
 // The contraction is issued as scores^T = Q K^T: the group's queries (zero padded to 64
 // rows) are the A operand and the key tile, exactly as TMA lands it, is the B operand
 // (N = keys of the tile).  The tensor core fetches B rows twice as fast as A rows, which
@@ -101,6 +229,13 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_kv = p.n_kv_heads, batch = p.batch, G = p.group;
 
+  // ---- clear this CTA's slice of the workspace head (counters, histograms, status word)
+  {
+    uint4* z = reinterpret_cast<uint4*>(p.status);
+    const size_t n16 = p.zero_bytes / 16;
+    for (size_t i = (size_t)blockIdx.x * kScoreThreads + tid; i < n16; i += (size_t)gridDim.x * kScoreThreads)
+      z[i] = make_uint4(0, 0, 0, 0);
+  }
   // ---- tiles per sequence -> prefix in shared memory
   {
     const int per = (batch + kScoreThreads - 1) / kScoreThreads;
@@ -318,17 +453,24 @@ cudaError_t launch_score(const Problem& p, const CUtensorMap& tm, int n_sm, cuda
 constexpr int kHistThreads = 512;
 constexpr int kHistChunk = 16384;                       // scores per CTA
 
-__global__ void __launch_bounds__(kHistThreads) hist_kernel(const Problem p) {
+__global__ void __launch_bounds__(kHistThreads) hist_kernel(const Problem p, const int n_chunk_ctas) {
   __shared__ unsigned h[kHistBins];
   __shared__ int scratch[40];
   __shared__ int s_last;
   const int b = blockIdx.z, hq = blockIdx.y, tid = threadIdx.x;
   const int row = b * p.n_q_heads + hq;
+  const int spare = p.with_phi ? 1 : 0;        // CTA 0 of a head does feature work, the others take chunks
+  if ((int)blockIdx.x < spare) {
+    // query log-features, and (once per KV head) the W_k split
+    phi_q_stage1<kHistThreads>(p, row);
+    if (b == 0 && hq % p.group == 0 && !(p.flags & 1u)) wk_split_job<kHistThreads>(p, hq / p.group);
+    return;
+  }
   const int K = p.topk[b];
   if (K == 0) return;
   const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
   const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
-  const int chunk0 = blockIdx.x * kHistChunk;
+  const int chunk0 = ((int)blockIdx.x - spare) * kHistChunk;
   if (chunk0 >= n_mid) return;
   const int n_chunks = (n_mid + kHistChunk - 1) / kHistChunk;
   const float* srow = p.scores + score_row_base(p, b, hq, cu_b, len_b);
@@ -380,139 +522,35 @@ __global__ void __launch_bounds__(kHistThreads) hist_kernel(const Problem p) {
 }
 
 cudaError_t launch_hist(const Problem& p, int max_mid, cudaStream_t st) {
-  if (max_mid <= 0) return cudaSuccess;
-  dim3 grid((max_mid + kHistChunk - 1) / kHistChunk, p.n_q_heads, p.batch);
-  hist_kernel<<<grid, kHistThreads, 0, st>>>(p);
+  const int n_chunk_ctas = max_mid > 0 ? (max_mid + kHistChunk - 1) / kHistChunk : 0;
+  const int extra = p.with_phi ? 1 : 0;
+  if (n_chunk_ctas + extra == 0) return cudaSuccess;
+  dim3 grid(n_chunk_ctas + extra, p.n_q_heads, p.batch);
+  hist_kernel<<<grid, kHistThreads, 0, st>>>(p, n_chunk_ctas);
   return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------ compaction against the threshold bin
-constexpr int kCompThreads = 256;
-constexpr int kCompPerWarp = kCompactChunk / (kCompThreads / 32);   // 512 scores per warp
-constexpr int kCompIters = kCompPerWarp / 32;                        // 16
-
-// Query-side work that does not depend on the selection (Sec. 4.1, Sec. 4.3): the
-// log-features a_q = W_q q + b_q - gamma_q |q|^2, kept as w = exp(a_q - m_q) and m_q so
-// that tiny features cannot underflow the merge, and the unsubtracted residual terms
-// S_M w (d values) and w . u_M.  Row layout of p.aq: [0, r) w, [r] m_q, [r+1] w . u_M,
-// [r+4, r+4+d) S_M w.
-__device__ void phi_q_job(const Problem& p, int row, int hq, int b) {
-  __shared__ float s_q[128];
-  __shared__ float s_a[128];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int D = p.head_dim, r = p.n_feat;
-  float* aq = p.aq + (size_t)row * (r + D + 4);
-  const __nv_bfloat16* qp = p.q + (size_t)row * D;
-  const float* W = p.w_q + (size_t)hq * r * D;
-  for (int c = tid; c < D; c += kCompThreads) s_q[c] = __bfloat162float(qp[c]);
-  __syncthreads();
-  float qn = 0.f;
-  for (int c = lane; c < D; c += 32) qn = fmaf(s_q[c], s_q[c], qn);
-  qn = warp_sum(qn);
-  // each warp owns r/8 feature rows: every lane loads its float4 of every row first (all
-  // loads in flight), then the dot products are reduced across the warp
-  constexpr int NW = kCompThreads / 32;
-  constexpr int MAXR = 128 / NW;                      // rows per warp at r = 128
-  const int rows_w = r / NW;
-  float part[MAXR];
-  const bool active = lane * 4 < D;
-#pragma unroll
-  for (int i = 0; i < MAXR; ++i) {
-    part[i] = 0.f;
-    if (i < rows_w && active) {
-      const float4 w4 = __ldg(reinterpret_cast<const float4*>(W + (size_t)(warp * rows_w + i) * D + lane * 4));
-      part[i] = w4.x * s_q[lane * 4] + w4.y * s_q[lane * 4 + 1] + w4.z * s_q[lane * 4 + 2] + w4.w * s_q[lane * 4 + 3];
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < MAXR; ++i) {
-    const float a = warp_sum(part[i]);
-    if (i < rows_w && lane == 0) {
-      const int j = warp * rows_w + i;
-      s_a[j] = a + p.b_q[(size_t)hq * r + j] - p.gamma_q * qn;
-    }
-  }
-  __syncthreads();
-  if (tid < 32) {
-    float m = -INFINITY;
-    for (int j = tid; j < r; j += 32) m = fmaxf(m, s_a[j]);
-    m = warp_max(m);
-    for (int j = tid; j < r; j += 32) { const float w = expf(s_a[j] - m); s_a[j] = w; aq[j] = w; }
-    if (tid == 0) aq[r] = m;
-  }
-  __syncthreads();
-  // S_M w: one warp per row of S (r floats = up to 32 lanes x float4), rows_d rows per warp
-  const int kvh = hq / p.group;
-  const float* Sg = p.S + ((size_t)b * p.n_kv_heads + kvh) * D * r;
-  const float* ug = p.u + ((size_t)b * p.n_kv_heads + kvh) * r;
-  const int rows_d = D / NW;
-  const bool act_r = lane * 4 < r;
-  float sp[MAXR];
-#pragma unroll
-  for (int i = 0; i < MAXR; ++i) {
-    sp[i] = 0.f;
-    if (i < rows_d && act_r) {
-      const float4 s4 = __ldg(reinterpret_cast<const float4*>(Sg + (size_t)(warp * rows_d + i) * r + lane * 4));
-      sp[i] = s4.x * s_a[lane * 4] + s4.y * s_a[lane * 4 + 1] + s4.z * s_a[lane * 4 + 2] + s4.w * s_a[lane * 4 + 3];
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < MAXR; ++i) {
-    const float a = warp_sum(sp[i]);
-    if (i < rows_d && lane == 0) aq[r + 4 + warp * rows_d + i] = a;
-  }
-  if (warp == 0) {
-    float a = 0.f;
-    for (int j = lane; j < r; j += 32) a = fmaf(ug[j], s_a[j], a);
-    a = warp_sum(a);
-    if (lane == 0) aq[r + 1] = a;
-  }
-}
-
-// W_k of one KV head (fp32 [r][d]) -> two bf16 images, hi = bf16(W) and lo = bf16(W - hi),
-// each laid out as the K-major, 128B-swizzled B operand of the feature recompute MMA:
-// [d/64 column blocks][r rows][128 bytes].
-__device__ void wk_split_job(const Problem& p, int kvh) {
-  const int D = p.head_dim, r = p.n_feat;
-  const float* W = p.w_k + (size_t)kvh * r * D;
-  unsigned char* hi = reinterpret_cast<unsigned char*>(p.wk_img + (size_t)kvh * 2 * r * D);
-  unsigned char* lo = hi + (size_t)r * D * 2;
-  const int cpr = D / 8;
-  for (int i = threadIdx.x; i < r * cpr; i += kCompThreads) {
-    const int row = i / cpr, c = i % cpr;
-    const float4 w0 = *reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8);
-    const float4 w1 = *reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8 + 4);
-    const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-    unsigned hw[4], lw[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(w[2 * e]), h1 = __float2bfloat16_rn(w[2 * e + 1]);
-      const __nv_bfloat16 l0 = __float2bfloat16_rn(w[2 * e] - __bfloat162float(h0));
-      const __nv_bfloat16 l1 = __float2bfloat16_rn(w[2 * e + 1] - __bfloat162float(h1));
-      hw[e] = (unsigned)__bfloat16_as_ushort(h0) | ((unsigned)__bfloat16_as_ushort(h1) << 16);
-      lw[e] = (unsigned)__bfloat16_as_ushort(l0) | ((unsigned)__bfloat16_as_ushort(l1) << 16);
-    }
-    const size_t off = (size_t)(c >> 3) * r * 128 + swz128(row, c & 7);
-    *reinterpret_cast<uint4*>(hi + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-    *reinterpret_cast<uint4*>(lo + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-  }
-}
+constexpr int kCompThreads = 512;
+constexpr int kCompPerWarp = kCompactChunk / (kCompThreads / 32);   // 1024 scores per warp
+constexpr int kCompIters = kCompPerWarp / 32;                        // 32
+static_assert(kCompIters == 32, "one bitmap word per lane");
 
 __global__ void __launch_bounds__(kCompThreads) compact_kernel(const Problem p, const int n_chunk_ctas) {
   const int b = blockIdx.z, hq = blockIdx.y;
   const int row = b * p.n_q_heads + hq;
-  if ((int)blockIdx.x >= n_chunk_ctas) {
-    // spare CTAs: feature-map work that does not depend on the scores
-    if ((int)blockIdx.x == n_chunk_ctas) phi_q_job(p, row, hq, b);
-    else if (b == 0 && hq % p.group == 0) wk_split_job(p, hq / p.group);
+  const int spare = p.with_phi ? 1 : 0;        // CTA 0 of a head does feature work, the others take chunks
+  if ((int)blockIdx.x < spare) {
+    phi_q_stage2<kCompThreads>(p, row);
     return;
   }
+  const int chunk = (int)blockIdx.x - spare;
   __shared__ int s_warp[kCompThreads / 32];
   const int K = p.topk[b];
   if (K == 0) return;
   const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
   const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
-  const int chunk0 = blockIdx.x * kCompactChunk;
+  const int chunk0 = chunk * kCompactChunk;
   if (chunk0 >= n_mid) return;
   const unsigned tb = (unsigned)p.rowinfo[row].x;
   const long long rbase = score_row_base(p, b, hq, cu_b, len_b);
@@ -555,7 +593,7 @@ __global__ void __launch_bounds__(kCompThreads) compact_kernel(const Problem p, 
     if (w < warp) off += c;
     total += c;
   }
-  if (threadIdx.x == 0) p.chunk_ncand[(size_t)row * p.max_chunks + blockIdx.x] = total;
+  if (threadIdx.x == 0) p.chunk_ncand[(size_t)row * p.max_chunks + chunk] = total;
   // ordered write: (warp, iteration, lane)
   int* out = p.cand + rbase + chunk0;
   const unsigned lt = (1u << lane) - 1u;
@@ -569,7 +607,7 @@ __global__ void __launch_bounds__(kCompThreads) compact_kernel(const Problem p, 
 
 cudaError_t launch_compact(const Problem& p, int max_mid, cudaStream_t st) {
   const int n_chunk_ctas = max_mid > 0 ? (max_mid + kCompactChunk - 1) / kCompactChunk : 0;
-  const int extra = p.with_phi ? 2 : 0;
+  const int extra = p.with_phi ? 1 : 0;
   if (n_chunk_ctas + extra == 0) return cudaSuccess;
   dim3 grid(n_chunk_ctas + extra, p.n_q_heads, p.batch);
   compact_kernel<<<grid, kCompThreads, 0, st>>>(p, n_chunk_ctas);
