@@ -226,11 +226,7 @@ def run_ours(args, rank, world, device):
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
 
-    ms = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([total_ms / args.steps, e2e_ms], world, device)
 
     ab = algorithmic_bytes(cfg, N, tmax, n_layers)
     peak, tf_burst, tf_sust, peak_kind = _peaks()
@@ -248,7 +244,7 @@ def run_ours(args, rank, world, device):
         "achieved_gbs": ab["total"] / (ms * 1e-3) / 1e9,
         "hbm_frac_of_measured_peak": ab["total"] / (ms * 1e-3) / 1e9 / peak,
         "algorithmic_bytes_per_step": ab["total"],
-        "steps_per_s_all_gpus": world * 1e3 / ms,
+        "steps_per_s_all_gpus": whole_job_steps_per_s(ms, world),
         "gpu_launches": args.steps * n_layers * 5,
         "e2e": {"value": e2e_ms * 1e3, "unit": "us/step", "h2d_bytes_per_step": q_stage.numel() * 2,
                 "d2h_bytes_per_step": y_host.numel() * 4},
@@ -265,6 +261,21 @@ def run_ours(args, rank, world, device):
                            "avg_launch_us": dom["avg_ms"] * 1e3}
         out["kernels_us_per_launch"] = {k: v["avg_ms"] * 1e3 for k, v in kt.items()}
     return out, (cfg, layers, phis, Ss, us, topk)
+
+
+def max_over_ranks(values, world, device=None):
+    """Replicas run independently (the path has no exchange step); a multi-rank number is the
+    slowest rank's.  Returns the element-wise maximum of `values` over all ranks."""
+    if world <= 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device or "cpu", dtype=torch.float64)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_steps_per_s(ms_per_step, world):
+    """Weak scaling: every rank decodes its own replica, so the job does `world` steps per step time."""
+    return world * 1e3 / ms_per_step
 
 
 def build_info(build_ms, n_layers, B, Hkv, n_mid, d, r, hbm_peak, tf_burst, tf_sust):
