@@ -380,11 +380,10 @@ tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc
   if (st != TKPHI_OK) return st;
   st = make_tensor_map(kv, kv->v, 128, sh.total_tokens, &tv);
   if (st != TKPHI_OK) return st;
-  cudaError_t e = cudaMemsetAsync(w, 0, L.zero_end, cs);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
+  cudaError_t e;
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_BUILD);
-    e = launch_build(p, tk, tv, cs);
+    e = launch_build(p, tk, tv, cs);      // clears the status word itself; needs no zeroed counters
   }
   if (e != cudaSuccess) return cuda_fail(e, "build launch");
   return TKPHI_OK;

@@ -18,9 +18,9 @@
 // Warp roles: 0 TMA producer, 1 MMA issuer, 2..9 feature warps, 10..13 key norms.
 // GEMM 1 of tile i+1 is issued before GEMM 2 of tile i, so the tensor pipe works while
 // the feature warps are busy.  Each CTA owns a contiguous range of tiles of one
-// (sequence, KV head) unit and writes one partial; the last CTA of the unit (atomic
-// ticket, no spinning) adds the partials in chunk order.  Every device-side wait is
-// bounded and reports through the status word.
+// (sequence, KV head) unit and writes one partial; a second small kernel adds the
+// partials in chunk order.  Every device-side wait is bounded and reports through the
+// status word.
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -81,8 +81,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   uint64_t* v_full = k_empty + KS;         // [VS]
   uint64_t* v_empty = v_full + VS;         // [VS] GEMM 2 is done with it
   uint64_t* d1_full = v_empty + VS;        // [2]  GEMM 1 accumulator complete
-  uint64_t* d1_empty = d1_full + 2;        // [2]  GEMM 2 has consumed the features stored over it
-  uint64_t* p_ready = d1_empty + 2;        // [2]  features stored to tensor memory
+  uint64_t* p_ready = d1_full + 2;         // [2]  features stored to tensor memory
   uint64_t* n_ready = p_ready + 2;         // [2]  key norms of the tile in shared memory
   uint64_t* d2_full = n_ready + 2;         // [1]  last GEMM 2 complete
   float* snorm = reinterpret_cast<float*>(bars + 32);        // [2][128]  -gamma log2e |k_t|^2, -inf if masked
@@ -90,7 +89,6 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   int* misc = reinterpret_cast<int*>(ucomb + 2 * 128);
   volatile int* s_abort = misc;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 1);
-  int* s_last = misc + 2;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.z, kvh = blockIdx.y, chunk = blockIdx.x;
@@ -100,6 +98,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
   float* S_out = p.S + (size_t)unit * D * R;
   float* u_out = p.u + (size_t)unit * R;
+  if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) *p.status = kStatusOk;
   if (n_mid == 0) {
     if (chunk == 0) {
       for (int i = tid; i < D * R; i += kBuildThreads) S_out[i] = 0.f;
@@ -120,7 +119,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 5); }
     for (int s = 0; s < VS; ++s) { mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&d1_full[s], 1); mbar_init(&d1_empty[s], 1); mbar_init(&p_ready[s], 8); mbar_init(&n_ready[s], 4);
+      mbar_init(&d1_full[s], 1); mbar_init(&p_ready[s], 8); mbar_init(&n_ready[s], 4);
     }
     mbar_init(d2_full, 1);
     mbar_fence_init();
@@ -215,12 +214,13 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
           umma_ts(tmem_base + kColD2, tmem_base + lo_col, bd, idesc2, 1u);
         }
         tc_commit(&v_empty[vs]);
-        tc_commit(&d1_empty[buf]);
       };
       for (int it = 0; it < n_my && ok; ++it) {
         const int buf = it & 1, ks = it % KS;
-        ok = mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort) &&
-             mbar_wait(&d1_empty[buf], ((uint32_t)(it >> 1) & 1u) ^ 1u, s_abort);
+        // No wait for GEMM 2 of tile it-2, whose A operand lives where this accumulator goes:
+        // MMAs issued by one thread execute in issue order, and the feature warps touch the
+        // buffer only after d1_full of this tile.
+        ok = mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort);
         if (!ok) break;
         tc_fence_after_sync();
         const uint64_t kd = k_d + (uint64_t)((ks * C::TILE) >> 4);
@@ -308,8 +308,9 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     bool ok = true;
     for (int it = 0; it < n_my && ok; ++it) {
       const int buf = it & 1, ks = it % KS;
+      // snorm[buf] was last read by the feature warps for tile it-2: wait for their p_ready
       ok = mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort) &&
-           mbar_wait(&d1_empty[buf], ((uint32_t)(it >> 1) & 1u) ^ 1u, s_abort);
+           mbar_wait(&p_ready[buf], ((uint32_t)(it >> 1) & 1u) ^ 1u, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       const unsigned char* tile = kring + ks * C::TILE;
@@ -345,18 +346,33 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   }
   float* part = p.partials + ((size_t)unit * p.chunks_per_unit + chunk) * ((size_t)D * R + R);
   if (tid < R) part[(size_t)D * R + tid] = ucomb[tid] + ucomb[128 + tid];
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) *s_last = (atomicAdd(&p.unit_counter[unit], 1u) == (unsigned)(n_chunks - 1));
-  __syncthreads();
-  if (!*s_last) return;
-  __threadfence();
-  // last CTA of the unit: add the chunk partials in chunk order
-  const float* parts = p.partials + (size_t)unit * p.chunks_per_unit * ((size_t)D * R + R);
-  for (int i = tid; i < D * R + R; i += kBuildThreads) {
+}
+
+// Adds the chunk partials of every unit in chunk order (fixed order: run-to-run identical).
+constexpr int kRedThreads = 256;
+constexpr int kRedBlocksPerUnit = 8;
+__global__ void __launch_bounds__(kRedThreads) build_reduce_kernel(const BuildProblem p) {
+  const int unit = blockIdx.y, b = unit / p.n_kv_heads;
+  const int D = p.head_dim, R = p.n_feat, n_out = D * R + R;
+  const long long len_b = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+  const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
+  if (n_mid == 0) return;                              // the build kernel wrote zeros
+  const int n_tiles = (n_mid + kBT - 1) / kBT;
+  const int n_chunks = n_tiles < p.chunks_per_unit ? n_tiles : p.chunks_per_unit;
+  const float* parts = p.partials + (size_t)unit * p.chunks_per_unit * n_out;
+  float* S_out = p.S + (size_t)unit * D * R;
+  float* u_out = p.u + (size_t)unit * R;
+  for (int i = blockIdx.x * kRedThreads + threadIdx.x; i < n_out; i += gridDim.x * kRedThreads) {
     float s = 0.f;
-#pragma unroll 4
-    for (int c = 0; c < n_chunks; ++c) s += __ldcg(parts + (size_t)c * ((size_t)D * R + R) + i);
+    int c = 0;
+    for (; c + 8 <= n_chunks; c += 8) {
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = __ldcg(parts + (size_t)(c + e) * n_out + i);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) s += v[e];
+    }
+    for (; c < n_chunks; ++c) s += __ldcg(parts + (size_t)c * n_out + i);
     if (i < D * R) S_out[i] = s; else u_out[i - D * R] = s;
   }
 }
@@ -373,6 +389,9 @@ static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, 
   }
   dim3 grid(p.chunks_per_unit, p.n_kv_heads, p.batch);
   build_kernel<D><<<grid, kBuildThreads, smem, st>>>(tk, tv, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  build_reduce_kernel<<<dim3(kRedBlocksPerUnit, p.n_kv_heads * p.batch), kRedThreads, 0, st>>>(p);
   return cudaGetLastError();
 }
 
