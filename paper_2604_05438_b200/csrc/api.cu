@@ -122,7 +122,7 @@ void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, W
   L->chunk_ncand = o;   o = align_up(o + sizeof(int) * (size_t)sh.rows * L->max_chunks, 256);
   L->wk_img = o;        o = align_up(o + (size_t)kv->n_kv_heads * 2 * kv->n_feat * kv->head_dim * 2, 1024);
   L->idx = o;           o = align_up(o + sizeof(int) * (size_t)sh.rows * (topk_max > 0 ? topk_max : 1), 256);
-  L->aq = o;            o = align_up(o + sizeof(float) * (size_t)sh.rows * (kv->n_feat + kv->head_dim + 4), 256);
+  L->aq = o;            o = align_up(o + sizeof(float) * (size_t)sh.rows * aq_stride(kv->n_feat, kv->head_dim), 256);
   int64_t max_support = (int64_t)kv->n_sink + kv->n_tail + topk_max;
   if (max_support > sh.max_len) max_support = sh.max_len;
   L->max_slices = (int)((max_support + kSlice - 1) / kSlice);

@@ -32,7 +32,6 @@ constexpr int kBuildTmemCols = 512;
 constexpr int kColD1 = 0;                // two GEMM-1 accumulators of 128 columns (Phi hi overwrites them)
 constexpr int kColD2 = 256;              // S^T accumulator, head_dim columns
 constexpr int kColLo = 384;              // Phi lo, 64 columns per buffer
-constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
 struct BuildCfg {
@@ -57,11 +56,6 @@ __device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[
       "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
       "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
-}
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
 }
 
 template <int D>

@@ -16,6 +16,7 @@ constexpr int kLowBits = 32 - kHistBits;      // bits refined inside the thresho
 constexpr int kMaxBatch = 1024;               // sequences per call
 constexpr int kSlice = 128;                   // exact-support tokens per CTA of the exact/residual kernel (= MMA M)
 constexpr int kCompactChunk = 16384;          // scores per CTA of the compaction kernel
+constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMaxChunks = 2048;              // compaction chunks per sequence the selection kernel can index
 
 // Device status word values (first word of the workspace).
@@ -55,7 +56,7 @@ struct Problem {
   int max_chunks;
   __nv_bfloat16* wk_img;           // [n_kv_heads][2][r*d] W_k split into bf16 hi / lo, stored as MMA operand tiles
   int* idx;                        // [rows][topk_max] ascending retrieved positions
-  float* aq;                       // [rows][n_feat + head_dim + 4]: exp(a_q - m_q), m_q, w.u_M, S_M w
+  float* aq;                       // [rows][aq_stride]: w = exp(a_q - m_q), m_q, w.u_M, S_M w, log2 w
   float* partials;                 // [rows][max_slices][partial_stride]
   int max_slices, partial_stride;
   float scale;                     // 1/sqrt(head_dim)
@@ -85,6 +86,8 @@ struct WsLayout {
   size_t b_partials; int chunk_len, chunks_per_unit;
 };
 
+// Row length of Problem::aq: [0, r) w; [r] m_q; [r+1] w.u_M; [r+4, r+4+d) S_M w; [r+4+d, 2r+4+d) log2 w.
+__host__ __device__ inline int aq_stride(int r, int d) { return 2 * r + d + 4; }
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // keys per TMA tile of the scoring kernel (32 KB of bf16 rows)
 __host__ __device__ inline int score_tile_keys(int head_dim) { return head_dim == 64 ? 256 : 128; }

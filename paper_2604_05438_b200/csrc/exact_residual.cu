@@ -36,11 +36,14 @@ struct ExSmem {
   static constexpr int KV_BOX = kSlice * 128;                 // bytes of one 64-dim column block of k or v
   static constexpr int W_BOX = R * 128;
   static constexpr size_t kt = 0;                             // bf16 k tile  [BOXES][128][128 B]
-  static constexpr size_t vt = kt + (size_t)BOXES * KV_BOX;   // bf16 v tile
-  static constexpr size_t whi = vt + (size_t)BOXES * KV_BOX;  // bf16 W_k hi  [BOXES][R][128 B]
+  static constexpr size_t whi = kt + (size_t)BOXES * KV_BOX;  // bf16 W_k hi  [BOXES][R][128 B]
   static constexpr size_t wlo = whi + (size_t)BOXES * W_BOX;
-  static constexpr size_t small = wlo + (size_t)BOXES * W_BOX;
-  // small: bars[2] (16 B), tok[128] int, isret[128] int, wgt[128], zt[128], qf[D], phiq[R], bk[R],
+  // the v tile takes over the W_k region once the MMAs have read it (the v rows wait in
+  // registers until then), which keeps the CTA small enough for two per SM
+  static constexpr size_t vt = whi;
+  static constexpr size_t w_bytes = 2 * (size_t)BOXES * W_BOX, v_bytes = (size_t)BOXES * KV_BOX;
+  static constexpr size_t small = whi + (w_bytes > v_bytes ? w_bytes : v_bytes);
+  // small: bars[2] (16 B), tok[128] int, isret[128] int, wgt[128], zt[128], qf[D], cj[R], spare[R],
   //        red[4*D], misc[16]
   static constexpr size_t total = small + 16 + 4 * (4 * kSlice + D + 2 * R + 4 * D + 16);
 };
@@ -59,9 +62,8 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   float* wgt = reinterpret_cast<float*>(isret + kSlice);
   float* zt = wgt + kSlice;
   float* qf = zt + kSlice;
-  float* phiq = qf + D;
-  float* bk = phiq + R;
-  float* red = bk + R;
+  float* cj = qf + D;               // log2 w_j + b_k[j] log2 e
+  float* red = cj + 2 * R;
   float* misc = red + 4 * D;
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 12);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 13);
@@ -109,10 +111,8 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   }
   for (int c = tid; c < D; c += kExThreads) qf[c] = __bfloat162float(p.q[(size_t)row * D + c]);
   if (do_phi) {
-    for (int j = tid; j < R; j += kExThreads) {
-      phiq[j] = p.aq[(size_t)row * (R + D + 4) + j];
-      bk[j] = p.b_k[(size_t)kvh * R + j];
-    }
+    for (int j = tid; j < R; j += kExThreads)
+      cj[j] = p.aq[(size_t)row * aq_stride(R, D) + R + 4 + D + j] + p.b_k[(size_t)kvh * R + j] * kLog2e;
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -125,18 +125,22 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   }
 
   // ---- 2. gather rows into swizzled tiles: v always; k for anchors (scores) and, with phi,
-  // retrieved rows.  Sixteen-byte asynchronous copies, all in flight at once.
-  constexpr int CPR = D / 8;                 // 16-byte chunks per row
-  for (int i = tid; i < kSlice * CPR; i += kExThreads) {
+  // retrieved rows.  Sixteen-byte copies, all in flight at once: k asynchronously into its tile,
+  // v into registers (its tile reuses the W_k region later).
+  constexpr int CPR = D / 8;                 // 16-byte chunks per row = copies per thread
+  uint4 vreg[CPR];
+#pragma unroll
+  for (int n = 0; n < CPR; ++n) {
+    const int i = tid + n * kExThreads;
     const int t = i / CPR, c = i % CPR;
     const int ti = tok[t];
     const uint32_t off = (c >> 3) * L::KV_BOX + swz128(t, c & 7);
+    vreg[n] = make_uint4(0, 0, 0, 0);
     if (ti >= 0) {
-      cp_async_16(vt + off, vbase + (long long)ti * p.stride_token + c * 8);
+      vreg[n] = __ldg(reinterpret_cast<const uint4*>(vbase + (long long)ti * p.stride_token + c * 8));
       if (!isret[t] || do_phi) cp_async_16(kt + off, kbase + (long long)ti * p.stride_token + c * 8);
       else *reinterpret_cast<uint4*>(kt + off) = make_uint4(0, 0, 0, 0);
     } else {
-      *reinterpret_cast<uint4*>(vt + off) = make_uint4(0, 0, 0, 0);
       *reinterpret_cast<uint4*>(kt + off) = make_uint4(0, 0, 0, 0);
     }
   }
@@ -198,21 +202,30 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   float z_t = 0.f;
   if (has_ret) {
     ok = mbar_wait(&bars[1], 0, s_abort);
-    ok = __syncthreads_and(ok ? 1 : 0) != 0;
-    if (ok) {
-      tc_fence_after_sync();
-      const uint32_t tmem_d = *s_tmem;
-      const float shift = -p.gamma_k * kn;
+    ok = __syncthreads_and(ok ? 1 : 0) != 0;       // the MMAs are done: W_k tiles are free
+  }
+  // the v rows move from registers into their tile (over the W_k region)
 #pragma unroll
-      for (int c4 = 0; c4 < R / 32; ++c4) {
-        float v[32];
-        tmem_ld_x32(tmem_addr(tmem_d, warp * 32, c4 * 32), v);
-        tc_wait_ld();
+  for (int n = 0; n < CPR; ++n) {
+    const int i = tid + n * kExThreads;
+    const int t = i / CPR, c = i % CPR;
+    *reinterpret_cast<uint4*>(vt + (c >> 3) * L::KV_BOX + swz128(t, c & 7)) = vreg[n];
+  }
+  if (has_ret && ok) {
+    tc_fence_after_sync();
+    const uint32_t tmem_d = *s_tmem;
+    // z = 2^(-gamma log2e |k|^2) * sum_j 2^(acc_j + c_j): four partial sums in a fixed order
+    float zp[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int j = 0; j < 32; ++j) z_t = fmaf(phiq[c4 * 32 + j], __expf(v[j] + bk[c4 * 32 + j] + shift), z_t);
-      }
-      if (!isret[tid]) z_t = 0.f;
+    for (int c4 = 0; c4 < R / 32; ++c4) {
+      float v[32];
+      tmem_ld_x32(tmem_addr(tmem_d, warp * 32, c4 * 32), v);
+      tc_wait_ld();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) zp[j & 3] += ex2_approx(v[j] + cj[c4 * 32 + j]);
     }
+    z_t = ((zp[0] + zp[1]) + (zp[2] + zp[3])) * ex2_approx(-p.gamma_k * kLog2e * kn);
+    if (!isret[tid]) z_t = 0.f;
   }
   zt[tid] = z_t;
   __syncthreads();
@@ -224,14 +237,18 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
     const int dv = tid % D, tg = tid / D;
     const unsigned char* vcol = vt + (dv >> 6) * L::KV_BOX + (dv & 7) * 2;
     const uint32_t ch = (dv & 63) >> 3;
-    float nu = 0.f, zv = 0.f;
-#pragma unroll 8
-    for (int t = tg * TPV; t < (tg + 1) * TPV; ++t) {
-      const unsigned short raw = *reinterpret_cast<const unsigned short*>(vcol + swz128(t, ch));
-      const float x = __uint_as_float((unsigned)raw << 16);
-      nu = fmaf(wgt[t], x, nu);
-      zv = fmaf(zt[t], x, zv);
+    float nu0 = 0.f, nu1 = 0.f, zv0 = 0.f, zv1 = 0.f;      // even / odd tokens, added in a fixed order
+#pragma unroll 4
+    for (int t = tg * TPV; t < (tg + 1) * TPV; t += 2) {
+      const unsigned short r0 = *reinterpret_cast<const unsigned short*>(vcol + swz128(t, ch));
+      const unsigned short r1 = *reinterpret_cast<const unsigned short*>(vcol + swz128(t + 1, ch));
+      const float x0 = __uint_as_float((unsigned)r0 << 16), x1 = __uint_as_float((unsigned)r1 << 16);
+      nu0 = fmaf(wgt[t], x0, nu0);
+      zv0 = fmaf(zt[t], x0, zv0);
+      nu1 = fmaf(wgt[t + 1], x1, nu1);
+      zv1 = fmaf(zt[t + 1], x1, zv1);
     }
+    const float nu = nu0 + nu1, zv = zv0 + zv1;
     red[tg * 2 * D + dv] = nu;
     red[tg * 2 * D + D + dv] = zv;
   }
@@ -312,7 +329,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   float y = 0.f, yR = 0.f, logZR = -INFINITY, Mx = m_E;
   if (p.with_phi) {
     // S_M phi_q and phi_q . u_M (in units of exp(m_q)) were prepared alongside phi_q
-    const float* aqr = p.aq + (size_t)row * (R + D + 4);
+    const float* aqr = p.aq + (size_t)row * aq_stride(R, D);
     const float m_q = aqr[R];
     const float Zt = aqr[R + 1] - zs;                      // Z_hat_R / exp(m_q)
     if (Zt > 0.f) {

@@ -83,7 +83,7 @@ __device__ __forceinline__ void cursor_next(TileCursor& c, const int* pre, int b
 // Query-side quantities (Sec. 4.1, Sec. 4.3): a_q = W_q q + b_q - gamma_q |q|^2, kept as
 // w = exp(a_q - m_q) and m_q so that tiny features cannot underflow the merge, and the
 // unsubtracted residual terms S_M w (d values) and w . u_M.  Row layout of p.aq:
-// [0, r) w, [r] m_q, [r+1] w . u_M, [r+4, r+4+d) S_M w.
+// [0, r) w, [r] m_q, [r+1] w . u_M, [r+4, r+4+d) S_M w, [r+4+d, 2r+4+d) log2 w.
 
 // Stage 1, by all NT threads of a CTA: w and m_q of query row `row`.
 template <int NT>
@@ -93,7 +93,7 @@ __device__ void phi_q_stage1(const Problem& p, int row) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int D = p.head_dim, r = p.n_feat;
   const int hq = row % p.n_q_heads;
-  float* aq = p.aq + (size_t)row * (r + D + 4);
+  float* aq = p.aq + (size_t)row * aq_stride(r, D);
   const __nv_bfloat16* qp = p.q + (size_t)row * D;
   const float* W = p.w_q + (size_t)hq * r * D;
   for (int c = tid; c < D; c += NT) s_q[c] = __bfloat162float(qp[c]);
@@ -129,7 +129,10 @@ __device__ void phi_q_stage1(const Problem& p, int row) {
   float m = -INFINITY;
   for (int j = lane; j < r; j += 32) m = fmaxf(m, s_a[j]);
   m = warp_max(m);                                    // every warp computes the same maximum
-  if (tid < r) aq[tid] = expf(s_a[tid] - m);
+  if (tid < r) {
+    aq[tid] = expf(s_a[tid] - m);
+    aq[r + 4 + D + tid] = (s_a[tid] - m) * kLog2e;     // the same weight in the log2 domain
+  }
   if (tid == 0) aq[r] = m;
 }
 
@@ -140,7 +143,7 @@ __device__ void phi_q_stage2(const Problem& p, int row) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int D = p.head_dim, r = p.n_feat;
   const int b = row / p.n_q_heads, hq = row % p.n_q_heads, kvh = hq / p.group;
-  float* aq = p.aq + (size_t)row * (r + D + 4);
+  float* aq = p.aq + (size_t)row * aq_stride(r, D);
   const float* Sg = p.S + ((size_t)b * p.n_kv_heads + kvh) * D * r;
   const float* ug = p.u + ((size_t)b * p.n_kv_heads + kvh) * r;
   constexpr int NW = NT / 32;
@@ -171,7 +174,8 @@ __device__ void phi_q_stage2(const Problem& p, int row) {
   }
 }
 
-// W_k of one KV head (fp32 [r][d]) -> two bf16 images, hi = bf16(W) and lo = bf16(W - hi),
+// W_k of one KV head (fp32 [r][d]), scaled by log2 e so that the recomputed exponents feed
+// exp2 directly -> two bf16 images, hi = bf16(W) and lo = bf16(W - hi),
 // each laid out as the K-major, 128B-swizzled B operand of the feature recompute MMA:
 // [d/64 column blocks][r rows][128 bytes].  By all NT threads of a CTA.
 template <int NT>
@@ -186,7 +190,8 @@ __device__ void wk_split_job(const Problem& p, int kvh) {
     const int row = i / cpr, c = i % cpr;
     const float4 w0 = __ldg(reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8));
     const float4 w1 = __ldg(reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8 + 4));
-    const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+    const float w[8] = {w0.x * kLog2e, w0.y * kLog2e, w0.z * kLog2e, w0.w * kLog2e,
+                        w1.x * kLog2e, w1.y * kLog2e, w1.z * kLog2e, w1.w * kLog2e};
     unsigned hw[4], lw[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {

@@ -61,6 +61,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // ------------------------------------------------------------------ proxies and copies
 // Makes shared-memory writes of ordinary stores visible to the async proxy (TMA,
 // tcgen05.mma operand reads).
