@@ -58,6 +58,8 @@ tkphi_status validate_kv(const tkphi_kv_desc* kv, Shape* sh, bool need_data) {
   }
   sh->total_tokens = cu[kv->batch];
   sh->rows = kv->batch * kv->n_q_heads;
+  if ((long long)sh->rows + (sh->rows + kv->n_kv_heads + 7) / 8 > 65535)
+    return fail(TKPHI_ERR_UNSUPPORTED, "batch * n_q_heads = %d is too large for one call", sh->rows);
   sh->units = kv->batch * kv->n_kv_heads;
   if (need_data) {
     if (!kv->cu_seqlens_dev) return fail(TKPHI_ERR_INVALID_ARG, "cu_seqlens_dev is NULL");
@@ -300,20 +302,10 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
   }
   {
-    ScopedSpan sp(cs, TKPHI_KERNEL_HIST);
-    e = launch_hist(p, sh.score_tiles > 0 ? sh.max_mid : 0, cs);
-  }
-  if (e != cudaSuccess) return cuda_fail(e, "hist launch");
-  {
-    ScopedSpan sp(cs, TKPHI_KERNEL_COMPACT);
-    e = launch_compact(p, sh.score_tiles > 0 ? sh.max_mid : 0, cs);
-  }
-  if (e != cudaSuccess) return cuda_fail(e, "compact launch");
-  {
     ScopedSpan sp(cs, TKPHI_KERNEL_FINALIZE_SELECT);
-    e = launch_finalize_select(p, cs);
+    e = launch_select(p, cs);
   }
-  if (e != cudaSuccess) return cuda_fail(e, "finalize_select launch");
+  if (e != cudaSuccess) return cuda_fail(e, "select launch");
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_EXACT_RESIDUAL);
     e = launch_exact_residual(p, cs);

@@ -168,6 +168,7 @@ __device__ __forceinline__ long long bitmap_row_base(const Problem& p, int b, in
 // Each returns cudaGetLastError() after enqueuing on `stream`.
 cudaError_t launch_score(const Problem& p, const CUtensorMap& tmap_k, int n_sm, cudaStream_t stream);
 cudaError_t launch_hist(const Problem& p, int max_mid, cudaStream_t stream);
+cudaError_t launch_select(const Problem& p, cudaStream_t stream);
 cudaError_t launch_compact(const Problem& p, int max_mid, cudaStream_t stream);
 cudaError_t launch_finalize_select(const Problem& p, cudaStream_t stream);
 cudaError_t launch_exact_residual(const Problem& p, cudaStream_t stream);

@@ -1,0 +1,317 @@
+// Exact Top-K selection over the score rows (exhaustive Top-K control selector, Sec. 5.1;
+// ties broken towards the lower index) in ONE kernel: a thread-block cluster of eight CTAs
+// per query head.
+//
+// Each CTA owns a contiguous eighth of the head's mid-region; each warp a contiguous
+// 1024-score run of it, read coalesced (lane l, step i -> element 32 i + l), so that
+// (CTA, round, warp, step, lane) order is index order.  For sequences of up to 131072
+// mid-region keys every CTA keeps its 16384 order-preserving score keys in shared memory
+// and the row is read from L2 exactly once (the loops over a thread's 32 keys stay rolled:
+// straight-line code that runs once is bound by instruction fetch, not by its work).  The exact K-th largest key is found by radix
+// selection over 12 + 10 + 10 bits: every CTA builds a local histogram in shared memory
+// and adds its non-zero bins into the accumulator of every CTA through distributed shared
+// memory; every CTA then walks its own copy of the accumulator.  Positions above the
+// threshold, and as many threshold ties as are still needed in index order, are then
+// written straight to their slot of the ascending index list: offsets come from warp
+// ballots, a scan over the warps of a CTA, and per-CTA totals exchanged through
+// distributed shared memory.  CTAs of a cluster only meet at hardware cluster barriers
+// (no flag spinning, no global scratch, nothing to clear between calls).
+//
+// Extra clusters of the same launch do the work that depends only on the call's inputs
+// (query-side features, W_k operand split), off the critical path.
+#include "common.cuh"
+#include "sm100.cuh"
+#include "feature_jobs.cuh"
+
+#include <cooperative_groups.h>
+
+namespace cg = cooperative_groups;
+
+namespace tkphi {
+
+constexpr int kSelThreads = 512;
+constexpr int kSelPer = 32;                              // scores per thread and round
+constexpr int kSelChunk = kSelThreads * kSelPer;         // 16384 scores per CTA and round
+constexpr int kSelCluster = 8;
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kRefBins = 1024;                           // two refinement digits of 10 bits
+
+struct SelShared {
+  unsigned hist[kHistBins];      // local 12-bit histogram
+  unsigned acc[kHistBins];       // the cluster's 12-bit histogram (every CTA receives every CTA's bins)
+  unsigned h1[kRefBins];         // local refinement histogram
+  unsigned acc1[kRefBins];       // the cluster's histogram of refinement digit 1
+  unsigned acc2[kRefBins];       // ... of refinement digit 2
+  int scratch[40];
+  int res[4];                    // result of a histogram walk: digit, count above it, count in it
+  int tot[2 * kSelCluster];      // per CTA: selected-for-sure count, tie count
+  int wdef[kSelWarps], wtie[kSelWarps];
+};
+
+// Walks an n-bin histogram (n = NB, a multiple of 512) from the top and finds the bin at
+// which the cumulative count reaches `need`; res = {bin, count above it, count in it}.
+// All 512 threads of the CTA call it.
+template <int NB>
+__device__ void walk_from_top(const unsigned* h, int need, int* res, int* scratch) {
+  constexpr int BPT = NB / kSelThreads;
+  const int tid = threadIdx.x;
+  unsigned loc[BPT];
+  int lsum = 0;
+#pragma unroll
+  for (int i = 0; i < BPT; ++i) { loc[i] = h[tid * BPT + i]; lsum += (int)loc[i]; }
+  int total;
+  const int excl = block_exclusive_scan(lsum, scratch, &total);
+  const int above = total - excl - lsum;                   // elements in bins above this thread's range
+  if (above < need && need <= above + lsum) {
+    int cum = above;
+#pragma unroll
+    for (int i = BPT - 1; i >= 0; --i) {
+      if (cum < need && need <= cum + (int)loc[i]) { res[0] = tid * BPT + i; res[1] = cum; res[2] = (int)loc[i]; }
+      cum += (int)loc[i];
+    }
+  }
+  __syncthreads();
+}
+
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads, 2)
+select_kernel(const Problem p, const int n_rows) {
+  __shared__ SelShared sm;
+  extern __shared__ __align__(16) unsigned keys_s[];       // [kSelPer][kSelThreads]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if ((int)blockIdx.y >= n_rows) {
+    // ---- feature clusters: one task per CTA (query rows first, then KV heads)
+    const int task = ((int)blockIdx.y - n_rows) * kSelCluster + (int)blockIdx.x;
+    if (task < n_rows) {
+      phi_q_stage1<kSelThreads>(p, task);
+      __threadfence_block();
+      __syncthreads();
+      phi_q_stage2<kSelThreads>(p, task);
+    } else if (task < n_rows + p.n_kv_heads && !(p.flags & 1u)) {
+      wk_split_job<kSelThreads>(p, task - n_rows);
+    }
+    return;
+  }
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const int row = blockIdx.y, b = row / p.n_q_heads, hq = row % p.n_q_heads;
+  const int K = p.topk[b];
+  int* out = p.idx + (size_t)row * p.topk_max;
+  int* out2 = p.idx_out ? p.idx_out + (size_t)row * p.topk_max : nullptr;
+  if (out2 && rank == 0)
+    for (int i = K + tid; i < p.topk_max; i += kSelThreads) out2[i] = -1;
+  if (K == 0) return;                                      // the same for all CTAs of the cluster
+
+  const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
+  const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
+  const float* srow = p.scores + score_row_base(p, b, hq, cu_b, len_b);
+  const int n_chunks = (n_mid + kSelChunk - 1) / kSelChunk;
+  const int rounds = (n_chunks + kSelCluster - 1) / kSelCluster;      // per CTA
+  const bool resident = rounds == 1;                       // the keys stay in shared memory
+  const unsigned low_mask = (1u << kLowBits) - 1u;
+
+  // Order-preserving keys of this thread's 32 scores of round k go to shared memory
+  // (element i at keys[i * 512]); bit i of vmask <=> score i lies inside the row.
+  unsigned* keys = keys_s + tid;
+  unsigned vmask = 0;
+  auto load_round = [&](int k) {
+    const int base = (rank * rounds + k) * kSelChunk + warp * (32 * kSelPer) + lane;
+    float sc[kSelPer];
+#pragma unroll
+    for (int i = 0; i < kSelPer; ++i) sc[i] = (base + i * 32 < n_mid) ? __ldcg(srow + base + i * 32) : 0.f;
+    vmask = 0;
+#pragma unroll
+    for (int i = 0; i < kSelPer; ++i) {
+      keys[i * kSelThreads] = ordered_key(sc[i]);
+      if (base + i * 32 < n_mid) vmask |= 1u << i;
+    }
+  };
+  // adds the non-zero bins of a local histogram into the accumulator of every CTA
+  auto push_all = [&](unsigned* local, unsigned* accum, int n_bins, bool clear) {
+    for (int i = tid; i < n_bins; i += kSelThreads) {
+      const unsigned c = local[i];
+      if (c) {
+#pragma unroll
+        for (int r = 0; r < kSelCluster; ++r) atomicAdd(cluster.map_shared_rank(accum, r) + i, c);
+        if (clear) local[i] = 0;
+      }
+    }
+  };
+
+  // ---- 12-bit histogram of the row, replicated in every CTA
+  for (int i = tid; i < kHistBins; i += kSelThreads) { sm.hist[i] = 0; sm.acc[i] = 0; }
+  for (int i = tid; i < kRefBins; i += kSelThreads) { sm.h1[i] = 0; sm.acc1[i] = 0; sm.acc2[i] = 0; }
+  __syncthreads();
+  for (int k = 0; k < rounds; ++k) {
+    load_round(k);
+#pragma unroll 4
+    for (int i = 0; i < kSelPer; ++i)
+      if ((vmask >> i) & 1u) atomicAdd(&sm.hist[keys[i * kSelThreads] >> kLowBits], 1u);
+  }
+  __syncthreads();
+  cluster.sync();                                          // every accumulator of the cluster is cleared
+  push_all(sm.hist, sm.acc, kHistBins, false);
+  cluster.sync();
+  walk_from_top<kHistBins>(sm.acc, K, sm.res, sm.scratch);
+  const unsigned tb = (unsigned)sm.res[0];                 // threshold bin
+  const int need = K - sm.res[1];                          // keys to take inside it, 1 <= need <= n_cand
+  const int n_cand = sm.res[2];
+  const bool refine = need < n_cand;                       // the same in every CTA
+
+  // bit i of smask: key i lies above the threshold bin; of cmask: inside it
+  unsigned smask = 0, cmask = 0;
+  auto classify_round = [&]() {
+    smask = 0; cmask = 0;
+#pragma unroll 4
+    for (int i = 0; i < kSelPer; ++i) {
+      const unsigned bin = keys[i * kSelThreads] >> kLowBits;
+      smask |= (bin > tb ? 1u : 0u) << i;
+      cmask |= (bin == tb ? 1u : 0u) << i;
+    }
+    smask &= vmask; cmask &= vmask;
+  };
+  if (resident) classify_round();
+
+  unsigned tau_low = 0;
+  int need_ties = n_cand;
+  if (refine) {
+    // ---- digit 1: bits 19..10 of the key among the keys of the threshold bin
+    for (int k = 0; k < rounds; ++k) {
+      if (!resident) { load_round(k); classify_round(); }
+      for (unsigned m = cmask; m; m &= m - 1) {
+        const int i = __ffs(m) - 1;
+        atomicAdd(&sm.h1[(keys[i * kSelThreads] & low_mask) >> 10], 1u);
+      }
+    }
+    __syncthreads();
+    push_all(sm.h1, sm.acc1, kRefBins, true);
+    cluster.sync();
+    walk_from_top<kRefBins>(sm.acc1, need, sm.res, sm.scratch);
+    const unsigned d1 = (unsigned)sm.res[0];
+    const int rem1 = need - sm.res[1];
+    __syncthreads();
+    // ---- digit 2: bits 9..0 among the keys whose digit 1 matches
+    for (int k = 0; k < rounds; ++k) {
+      if (!resident) { load_round(k); classify_round(); }
+      for (unsigned m = cmask; m; m &= m - 1) {
+        const int i = __ffs(m) - 1;
+        const unsigned low = keys[i * kSelThreads] & low_mask;
+        if ((low >> 10) == d1) atomicAdd(&sm.h1[low & (kRefBins - 1)], 1u);
+      }
+    }
+    __syncthreads();
+    push_all(sm.h1, sm.acc2, kRefBins, false);
+    cluster.sync();
+    walk_from_top<kRefBins>(sm.acc2, rem1, sm.res, sm.scratch);
+    tau_low = (d1 << 10) | (unsigned)sm.res[0];
+    need_ties = rem1 - sm.res[1];
+  }
+
+  // after this, smask: keys above the exact threshold; cmask: keys equal to it (without
+  // refinement the whole threshold bin counts as tied: all of it is taken)
+  auto finish_masks = [&]() {
+    if (!refine) return;
+    unsigned tie = 0;
+    for (unsigned m = cmask; m; m &= m - 1) {
+      const int i = __ffs(m) - 1;
+      const unsigned low = keys[i * kSelThreads] & low_mask;
+      if (low > tau_low) smask |= 1u << i;
+      else if (low == tau_low) tie |= 1u << i;
+    }
+    cmask = tie;
+  };
+  if (resident) finish_masks();
+
+  // ---- per-CTA totals, exchanged so that every CTA knows what the CTAs before it contribute
+  {
+    int n_sure = 0, n_tie = 0;
+    for (int k = 0; k < rounds; ++k) {
+      if (!resident) { load_round(k); classify_round(); finish_masks(); }
+      n_sure += __popc(smask);
+      n_tie += __popc(cmask);
+    }
+    n_sure = warp_sum_int(n_sure);
+    n_tie = warp_sum_int(n_tie);
+    if (lane == 0) { sm.wdef[warp] = n_sure; sm.wtie[warp] = n_tie; }
+    __syncthreads();
+    if (tid < kSelCluster) {
+      int a = 0, c = 0;
+      for (int w = 0; w < kSelWarps; ++w) { a += sm.wdef[w]; c += sm.wtie[w]; }
+      int* r = cluster.map_shared_rank(sm.tot, tid);
+      r[2 * rank] = a;
+      r[2 * rank + 1] = c;
+    }
+  }
+  cluster.sync();                                          // also the last access to another CTA's memory
+  int tie_base = 0, out_base = 0;                          // ties / selected positions before this CTA
+  for (int r = 0; r < rank; ++r) {
+    const int t = sm.tot[2 * r + 1];
+    int take = need_ties - tie_base;
+    take = take < 0 ? 0 : (take > t ? t : take);
+    out_base += sm.tot[2 * r] + take;
+    tie_base += t;
+  }
+
+  // ---- write the selected positions of this CTA in index order
+  for (int k = 0; k < rounds; ++k) {
+    if (!resident) { load_round(k); classify_round(); finish_masks(); }
+    const int w_sure = warp_sum_int(__popc(smask)), w_tie = warp_sum_int(__popc(cmask));
+    __syncthreads();                                       // wdef / wtie of the previous use are read
+    if (lane == 0) { sm.wdef[warp] = w_sure; sm.wtie[warp] = w_tie; }
+    __syncthreads();
+    int tie_run = tie_base, out_run = out_base;            // before this warp, then before this step
+    int r_tie = 0, r_sel = 0;                              // this round's totals
+    for (int w = 0; w < kSelWarps; ++w) {
+      const int t = sm.wtie[w];
+      int take = need_ties - (tie_base + r_tie);
+      take = take < 0 ? 0 : (take > t ? t : take);
+      if (w < warp) { tie_run += t; out_run += sm.wdef[w] + take; }
+      r_tie += t;
+      r_sel += sm.wdef[w] + take;
+    }
+    const unsigned lt = (1u << lane) - 1u;
+    const int pos0 = p.n_sink + (rank * rounds + k) * kSelChunk + warp * (32 * kSelPer) + lane;
+    if (w_sure + w_tie > 0) {                              // most warps of most rounds hold nothing
+#pragma unroll 2
+      for (int i = 0; i < kSelPer; ++i) {
+        const bool t = (cmask >> i) & 1u;
+        const unsigned sure_m = __ballot_sync(0xffffffffu, (smask >> i) & 1u);
+        const unsigned tie_m = __ballot_sync(0xffffffffu, t);
+        if ((sure_m | tie_m) == 0) continue;
+        int n_take = need_ties - tie_run;                  // ties of this step that are still admitted
+        const int nt = __popc(tie_m);
+        n_take = n_take < 0 ? 0 : (n_take > nt ? nt : n_take);
+        const bool taken = t && __popc(tie_m & lt) < n_take;
+        const unsigned sel = sure_m | __ballot_sync(0xffffffffu, taken);
+        if ((sel >> lane) & 1u) {
+          const int off = out_run + __popc(sel & lt);
+          if (off < K) {
+            out[off] = pos0 + i * 32;
+            if (out2) out2[off] = pos0 + i * 32;
+          }
+        }
+        out_run += __popc(sel);
+        tie_run += nt;
+      }
+    }
+    tie_base += r_tie;
+    out_base += r_sel;
+  }
+}
+
+cudaError_t launch_select(const Problem& p, cudaStream_t st) {
+  const int rows = p.batch * p.n_q_heads;
+  const int n_tasks = p.with_phi ? rows + p.n_kv_heads : 0;
+  const int feat_clusters = (n_tasks + kSelCluster - 1) / kSelCluster;
+  dim3 grid(kSelCluster, rows + feat_clusters, 1);
+  static bool configured = false;
+  constexpr size_t smem = sizeof(unsigned) * kSelChunk;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  select_kernel<<<grid, kSelThreads, smem, st>>>(p, rows);
+  return cudaGetLastError();
+}
+
+}  // namespace tkphi
