@@ -206,12 +206,12 @@ tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32
  */
 enum {
   TKPHI_KERNEL_SCORE = 0,           /* key scoring (streams the mid-region keys) */
-  TKPHI_KERNEL_COMPACT = 1,         /* bitmap and candidate lists against the threshold bin; phi_q; W_k split */
-  TKPHI_KERNEL_FINALIZE_SELECT = 2, /* exact threshold, ties, ascending index list */
+  TKPHI_KERNEL_RESERVED_1 = 1,
+  TKPHI_KERNEL_SELECT = 2,          /* exact Top-K over the score rows; query-side feature work */
   TKPHI_KERNEL_EXACT_RESIDUAL = 3,  /* exact branch, subtraction, residual, merge */
   TKPHI_KERNEL_BUILD = 4,           /* prefill summary build */
-  TKPHI_KERNEL_MEMSET = 5,          /* clearing counters and histograms */
-  TKPHI_KERNEL_HIST = 6,            /* score histogram and threshold bin */
+  TKPHI_KERNEL_MEMSET = 5,          /* clearing counters when there is nothing to score */
+  TKPHI_KERNEL_RESERVED_6 = 6,
   TKPHI_KERNEL_KINDS = 7
 };
 void tkphi_kernel_timing_enable(int32_t on);

@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = (
     "tkphi_build_summaries_static", "tkphi_static_last_error",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
-KERNEL_KINDS = ("score", "compact", "finalize_select", "exact_residual", "build", "memset", "hist")
+KERNEL_KINDS = ("score", "reserved_1", "select", "exact_residual", "build", "memset", "reserved_6")
 
 
 class TkphiError(RuntimeError):

@@ -90,9 +90,6 @@ tkphi_status validate_topk(const tkphi_kv_desc* kv, const int32_t* topk_host, in
     if (!allow_empty_support && topk_host[b] == 0 && kv->n_sink == 0 && kv->n_tail == 0)
       return fail(TKPHI_ERR_INVALID_ARG, "sequence %d has an empty exact support (no anchors, topk = 0)", b);
     if (topk_host[b] > 0) sh->score_tiles += (int64_t)kv->n_kv_heads * ((mid + tk - 1) / tk);
-    if (mid > (int64_t)kMaxChunks * kCompactChunk)
-      return fail(TKPHI_ERR_UNSUPPORTED, "sequence %d: mid-region of %lld tokens exceeds %lld", b, (long long)mid,
-                  (long long)kMaxChunks * kCompactChunk);
   }
   if (sh->score_tiles >= (1ll << 31)) return fail(TKPHI_ERR_UNSUPPORTED, "too many key tiles");
   return TKPHI_OK;
@@ -111,17 +108,9 @@ int n_sm_cached() {
 void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, WsLayout* L) {
   size_t o = 0;
   L->status = o;        o += 256;
-  L->unit_counter = o;  o = align_up(o + sizeof(unsigned) * sh.rows, 256);
   L->row_counter = o;   o = align_up(o + sizeof(unsigned) * sh.rows, 256);
-  L->hist = o;          o = align_up(o + sizeof(unsigned) * (size_t)sh.rows * kHistBins, 256);
   L->zero_end = o;
-  L->rowinfo = o;       o = align_up(o + sizeof(int4) * sh.rows, 256);
   L->scores = o;        o = align_up(o + sizeof(float) * (size_t)kv->n_q_heads * sh.total_tokens, 256);
-  const size_t bm_words = ((size_t)kv->n_q_heads * sh.total_tokens) / 32 + sh.rows + 2;
-  L->bm_sure = o;       o = align_up(o + 4 * bm_words, 256);
-  L->cand = o;          o = align_up(o + sizeof(int) * (size_t)kv->n_q_heads * sh.total_tokens, 256);
-  L->max_chunks = sh.max_mid > 0 ? (sh.max_mid + kCompactChunk - 1) / kCompactChunk : 1;
-  L->chunk_ncand = o;   o = align_up(o + sizeof(int) * (size_t)sh.rows * L->max_chunks, 256);
   L->wk_img = o;        o = align_up(o + (size_t)kv->n_kv_heads * 2 * kv->n_feat * kv->head_dim * 2, 1024);
   L->idx = o;           o = align_up(o + sizeof(int) * (size_t)sh.rows * (topk_max > 0 ? topk_max : 1), 256);
   L->aq = o;            o = align_up(o + sizeof(float) * (size_t)sh.rows * aq_stride(kv->n_feat, kv->head_dim), 256);
@@ -263,15 +252,8 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   }
   p.idx_out = idx_out; p.y_out = y_out; p.dbg_out = dbg_out; p.flags = flags; p.with_phi = with_phi ? 1 : 0;
   p.status = reinterpret_cast<int*>(w + L.status);
-  p.unit_counter = reinterpret_cast<unsigned*>(w + L.unit_counter);
   p.row_counter = reinterpret_cast<unsigned*>(w + L.row_counter);
-  p.rowinfo = reinterpret_cast<int4*>(w + L.rowinfo);
-  p.hist = reinterpret_cast<unsigned*>(w + L.hist);
   p.scores = reinterpret_cast<float*>(w + L.scores);
-  p.bm_sure = reinterpret_cast<unsigned*>(w + L.bm_sure);
-  p.cand = reinterpret_cast<int*>(w + L.cand);
-  p.chunk_ncand = reinterpret_cast<int*>(w + L.chunk_ncand);
-  p.max_chunks = L.max_chunks;
   p.wk_img = reinterpret_cast<__nv_bfloat16*>(w + L.wk_img);
   p.idx = reinterpret_cast<int*>(w + L.idx);
   p.aq = reinterpret_cast<float*>(w + L.aq);
@@ -284,9 +266,7 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   p.zero_bytes = L.zero_end;
   cudaError_t e;
   // The scoring kernel also clears the workspace counters; without keys to score a plain
-  // memset does.  The histogram and compaction kernels carry the query-side feature work
-  // on spare CTAs, so they are launched (possibly with no score chunks) whenever there are
-  // feature maps.
+  // memset does.  The selection kernel carries the query-side feature work on extra clusters.
   if (sh.score_tiles > 0) {
     CUtensorMap tm;
     st = make_tensor_map(kv, kv->k, score_tile_keys(kv->head_dim), sh.total_tokens, &tm);
@@ -302,7 +282,7 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
   }
   {
-    ScopedSpan sp(cs, TKPHI_KERNEL_FINALIZE_SELECT);
+    ScopedSpan sp(cs, TKPHI_KERNEL_SELECT);
     e = launch_select(p, cs);
   }
   if (e != cudaSuccess) return cuda_fail(e, "select launch");

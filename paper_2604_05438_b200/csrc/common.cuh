@@ -15,9 +15,7 @@ constexpr int kHistBins = 1 << kHistBits;     // bins of the fused first-pass hi
 constexpr int kLowBits = 32 - kHistBits;      // bits refined inside the threshold bin
 constexpr int kMaxBatch = 1024;               // sequences per call
 constexpr int kSlice = 128;                   // exact-support tokens per CTA of the exact/residual kernel (= MMA M)
-constexpr int kCompactChunk = 16384;          // scores per CTA of the compaction kernel
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kMaxChunks = 2048;              // compaction chunks per sequence the selection kernel can index
 
 // Device status word values (first word of the workspace).
 constexpr int kStatusOk = 0;
@@ -45,15 +43,8 @@ struct Problem {
   // workspace pieces (device pointers)
   int* status;                     // first word of the workspace
   size_t zero_bytes;               // head of the workspace that must be zero before the selection kernels
-  unsigned* unit_counter;          // [batch*n_q_heads] histogram-chunk tickets
   unsigned* row_counter;           // [batch*n_q_heads]
-  int4* rowinfo;                   // [rows]: x = threshold bin, y = count above, z = count in bin
-  unsigned* hist;                  // [rows][kHistBins]
   float* scores;                   // [n_q_heads * total_tokens]
-  unsigned* bm_sure;               // bitmap of selected mid positions (first: those above the threshold bin)
-  int* cand;                       // threshold-bin candidates (mid offsets), one segment per compaction chunk
-  int* chunk_ncand;                // [rows][max_chunks] candidates per chunk
-  int max_chunks;
   __nv_bfloat16* wk_img;           // [n_kv_heads][2][r*d] W_k split into bf16 hi / lo, stored as MMA operand tiles
   int* idx;                        // [rows][topk_max] ascending retrieved positions
   float* aq;                       // [rows][aq_stride]: w = exp(a_q - m_q), m_q, w.u_M, S_M w, log2 w
@@ -79,9 +70,9 @@ struct BuildProblem {
 
 // Host-side byte offsets of the workspace pieces.
 struct WsLayout {
-  size_t status, unit_counter, row_counter, hist, zero_end;
-  size_t rowinfo, scores, bm_sure, cand, chunk_ncand, wk_img, idx, aq, partials, total;
-  int max_slices, partial_stride, max_chunks;
+  size_t status, unit_counter, row_counter, zero_end;
+  size_t scores, wk_img, idx, aq, partials, total;
+  int max_slices, partial_stride;
   // build
   size_t b_partials; int chunk_len, chunks_per_unit;
 };
@@ -155,22 +146,14 @@ __device__ __forceinline__ int block_exclusive_scan(int x, int* scratch, int* to
 }
 
 // Offsets that follow from cu_seqlens alone (no per-call prefix arrays needed):
-// the score row of (b, hq) starts at element H_q*cu[b] + hq*L_b, and its bitmap
-// at word (that offset)/32 + row, which never overlaps the next row's words.
+// the score row of (b, hq) starts at element H_q*cu[b] + hq*L_b.
 __device__ __forceinline__ long long score_row_base(const Problem& p, int b, int hq, long long cu_b, long long len_b) {
   return (long long)p.n_q_heads * cu_b + (long long)hq * len_b;
 }
-__device__ __forceinline__ long long bitmap_row_base(const Problem& p, int b, int hq, long long cu_b, long long len_b) {
-  return (score_row_base(p, b, hq, cu_b, len_b) >> 5) + (long long)(b * p.n_q_heads + hq);
-}
-
 // ---------------------------------------------------------------- host launchers
 // Each returns cudaGetLastError() after enqueuing on `stream`.
 cudaError_t launch_score(const Problem& p, const CUtensorMap& tmap_k, int n_sm, cudaStream_t stream);
-cudaError_t launch_hist(const Problem& p, int max_mid, cudaStream_t stream);
 cudaError_t launch_select(const Problem& p, cudaStream_t stream);
-cudaError_t launch_compact(const Problem& p, int max_mid, cudaStream_t stream);
-cudaError_t launch_finalize_select(const Problem& p, cudaStream_t stream);
 cudaError_t launch_exact_residual(const Problem& p, cudaStream_t stream);
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, cudaStream_t stream);
 

@@ -96,8 +96,8 @@ def test_workspace_sizes_scale_with_the_problem(lib):
     a = lib.tkphi_workspace_bytes(C.byref(d1), t.ctypes.data, 40, T.WS_DECODE_STEP)
     b = lib.tkphi_workspace_bytes(C.byref(d2), t.ctypes.data, 40, T.WS_DECODE_STEP)
     assert 0 < a < b and a % 256 == 0
-    # scores (4 B), candidate list (4 B) and one bitmap bit per (query head, token) dominate the growth
-    assert abs((b - a) - 4096 * 32 * (8 + 0.125)) < 64 * 1024
+    # the fp32 score rows (4 B per query head and token) dominate the growth
+    assert abs((b - a) - 4096 * 32 * 4) < 64 * 1024
     assert lib.tkphi_workspace_bytes(C.byref(d1), None, 0, T.WS_BUILD) > 0
     assert lib.tkphi_workspace_bytes(C.byref(d1), None, 40, T.WS_DECODE_STEP) == 0     # topk_host required
     assert lib.tkphi_workspace_bytes(C.byref(d1), t.ctypes.data, 40, 9) == 0
