@@ -150,6 +150,20 @@ __device__ __forceinline__ int block_exclusive_scan(int x, int* scratch, int* to
 __device__ __forceinline__ long long score_row_base(const Problem& p, int b, int hq, long long cu_b, long long len_b) {
   return (long long)p.n_q_heads * cu_b + (long long)hq * len_b;
 }
+// Launch with programmatic stream serialization: the kernel may begin (up to its
+// pdl_wait()) while the previous kernel of the stream is still finishing.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---------------------------------------------------------------- host launchers
 // Each returns cudaGetLastError() after enqueuing on `stream`.
 cudaError_t launch_score(const Problem& p, const CUtensorMap& tmap_k, int n_sm, cudaStream_t stream);

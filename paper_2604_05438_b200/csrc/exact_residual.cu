@@ -70,6 +70,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.z, hq = blockIdx.y, slice = blockIdx.x;
+  pdl_launch_next();
   const int row = b * p.n_q_heads + hq, kvh = hq / p.group;
   const int K = p.topk[b];
   const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
@@ -97,6 +98,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
     *s_abort = 0;
   }
   if (has_ret && warp == 0) tmem_alloc(s_tmem, R);
+  pdl_wait();                                  // the index lists, features and score rows of the predecessors
   // ---- 1. token list of this slice
   {
     const int pi = slice * kSlice + tid;
@@ -365,8 +367,7 @@ static cudaError_t launch_ex_t(const Problem& p, cudaStream_t st) {
     configured = true;
   }
   dim3 grid(p.max_slices, p.n_q_heads, p.batch);
-  exact_residual_kernel<D, R><<<grid, kExThreads, smem, st>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(exact_residual_kernel<D, R>, grid, dim3(kExThreads), smem, st, p);
 }
 
 cudaError_t launch_exact_residual(const Problem& p, cudaStream_t st) {

@@ -88,14 +88,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_kv = p.n_kv_heads, batch = p.batch, G = p.group;
 
-  // ---- clear this CTA's slice of the workspace head (counters, histograms, status word)
-  {
-    uint4* z = reinterpret_cast<uint4*>(p.status);
-    const size_t n16 = p.zero_bytes / 16;
-    for (size_t i = (size_t)blockIdx.x * kScoreThreads + tid; i < n16; i += (size_t)gridDim.x * kScoreThreads)
-      z[i] = make_uint4(0, 0, 0, 0);
-  }
-  // ---- tiles per sequence -> prefix in shared memory
+  pdl_launch_next();
+  // ---- tiles per sequence -> prefix in shared memory (reads only the call's inputs)
   {
     const int per = (batch + kScoreThreads - 1) / kScoreThreads;
     const int b0 = tid * per;
@@ -130,6 +124,15 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
     *s_abort = 0;
   }
   if (warp == 1) tmem_alloc(s_tmem, kTmemCols);
+  // everything below touches the workspace, which kernels of the previous call may still use
+  pdl_wait();
+  // ---- clear this CTA's slice of the workspace head (counters, status word)
+  {
+    uint4* z = reinterpret_cast<uint4*>(p.status);
+    const size_t n16 = p.zero_bytes / 16;
+    for (size_t i = (size_t)blockIdx.x * kScoreThreads + tid; i < n16; i += (size_t)gridDim.x * kScoreThreads)
+      z[i] = make_uint4(0, 0, 0, 0);
+  }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -298,8 +301,7 @@ static cudaError_t launch_score_t(const Problem& p, const CUtensorMap& tm, int n
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  score_kernel<D><<<n_sm, kScoreThreads, smem, st>>>(tm, p);
-  return cudaGetLastError();
+  return launch_pdl(score_kernel<D>, dim3(n_sm), dim3(kScoreThreads), smem, st, tm, p);
 }
 
 cudaError_t launch_score(const Problem& p, const CUtensorMap& tm, int n_sm, cudaStream_t st) {

@@ -78,6 +78,8 @@ select_kernel(const Problem p, const int n_rows) {
   __shared__ SelShared sm;
   extern __shared__ __align__(16) unsigned keys_s[];       // [kSelPer][kSelThreads]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_next();
+  pdl_wait();                                              // score rows and workspace of the predecessors
   if ((int)blockIdx.y >= n_rows) {
     // ---- feature clusters: one task per CTA (query rows first, then KV heads)
     const int task = ((int)blockIdx.y - n_rows) * kSelCluster + (int)blockIdx.x;
@@ -310,8 +312,7 @@ cudaError_t launch_select(const Problem& p, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  select_kernel<<<grid, kSelThreads, smem, st>>>(p, rows);
-  return cudaGetLastError();
+  return launch_pdl(select_kernel, grid, dim3(kSelThreads), smem, st, p, rows);
 }
 
 }  // namespace tkphi
