@@ -46,7 +46,7 @@ def _peaks():
 
 # DRAM bytes per launch of the scoring kernel from the committed ncu capture of this kernel
 # (profiles/); None once the kernel has changed since the capture.
-SCORE_KERNEL_NCU_TRAFFIC_BYTES = None
+SCORE_KERNEL_NCU_TRAFFIC_BYTES = 268232960 + 11801856   # dram read + write, profiles/decode_kernels_c3_one_layer.md
 
 
 # --------------------------------------------------------------------------- clocks
@@ -92,7 +92,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            self._stop.wait(0.1)
+            self._stop.wait(0.01)
 
     def stop(self):
         self._stop.set()
@@ -195,7 +195,6 @@ def run_ours(args, rank, world, device):
         step(q_dev[s % n_q_sets])
         ev[s + 1].record()
     barrier()
-    clocks = sampler.stop()
     per_step = [ev[s].elapsed_time(ev[s + 1]) for s in range(args.steps)]
     total_ms = ev[0].elapsed_time(ev[args.steps])
     assert T.device_status(ws) == 0, "a device-side wait timed out"
@@ -225,6 +224,7 @@ def run_ours(args, rank, world, device):
         step_e2e(s)
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    clocks = sampler.stop()          # sampled over both timed regions (device-timed loop and end-to-end loop)
 
     ms, e2e_ms = max_over_ranks([total_ms / args.steps, e2e_ms], world, device)
 
@@ -399,12 +399,12 @@ def main():
             cfg = CONFIGS[args.config]
             n_layers = args.layers or cfg.n_layers
             N = args.seq_len or cfg.seq_len
-            smp = OracleSample(cfg, N, args.budget, 8, n_queries=4)
-            dts, ests = zip(*[smp.step(i) for i in range(4)])
+            smp = OracleSample(cfg, N, args.budget, 8, n_queries=16)
+            dts, ests = zip(*[smp.step(i) for i in range(16)])
             out["cpu_baseline"] = {
                 "value": statistics.mean(ests) * n_layers * 1e6, "unit": "us/step", "cores": smp.threads,
                 "kind": "oracle",
-                "sample": f"{len(smp.heads)} of {cfg.n_q_heads} query heads of one layer at full N={N}, 4 decode "
+                "sample": f"{len(smp.heads)} of {cfg.n_q_heads} query heads of one layer at full N={N}, 16 decode "
                           f"queries each ({sum(dts):.1f} s of oracle time), scaled by heads and {n_layers} layers; "
                           f"summaries prebuilt"}
         print(json.dumps(out), flush=True)

@@ -344,7 +344,6 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
 
 // Adds the chunk partials of every unit in chunk order (fixed order: run-to-run identical).
 constexpr int kRedThreads = 256;
-constexpr int kRedBlocksPerUnit = 8;
 __global__ void __launch_bounds__(kRedThreads) build_reduce_kernel(const BuildProblem p) {
   const int unit = blockIdx.y, b = unit / p.n_kv_heads;
   const int D = p.head_dim, R = p.n_feat, n_out = D * R + R;
@@ -385,7 +384,9 @@ static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, 
   build_kernel<D><<<grid, kBuildThreads, smem, st>>>(tk, tv, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  build_reduce_kernel<<<dim3(kRedBlocksPerUnit, p.n_kv_heads * p.batch), kRedThreads, 0, st>>>(p);
+  // one output per thread: every thread's loads of all chunk partials are in flight at once
+  const int n_out = p.head_dim * p.n_feat + p.n_feat;
+  build_reduce_kernel<<<dim3((n_out + kRedThreads - 1) / kRedThreads, p.n_kv_heads * p.batch), kRedThreads, 0, st>>>(p);
   return cudaGetLastError();
 }
 

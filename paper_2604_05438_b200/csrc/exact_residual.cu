@@ -97,8 +97,8 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
     mbar_fence_init();
     *s_abort = 0;
   }
-  if (has_ret && warp == 0) tmem_alloc(s_tmem, R);
   pdl_wait();                                  // the index lists, features and score rows of the predecessors
+  if (has_ret && warp == 0) tmem_alloc(s_tmem, R);   // after the wait: never hold columns a predecessor needs
   // ---- 1. token list of this slice
   {
     const int pi = slice * kSlice + tid;

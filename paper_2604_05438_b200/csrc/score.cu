@@ -3,7 +3,7 @@
 // The selection over the score rows is in select_cluster.cu.
 //
 //   score_kernel   streams the keys once.  A producer thread issues TMA loads of
-//                  128B-swizzled 32 KB key tiles into a 6-stage mbarrier ring; one thread
+//                  128B-swizzled 32 KB key tiles into a 3-stage mbarrier ring; one thread
 //                  issues tcgen05.mma with the key tile as an operand straight from shared
 //                  memory and the group's queries (zero padded) as the other, so the dot
 //                  products cost no issue slots of the CUDA cores; one warp reads the fp32
@@ -16,7 +16,7 @@ namespace tkphi {
 
 // ------------------------------------------------------------------ scoring
 constexpr int kScoreThreads = 96;         // warp 0: read-back, warp 1: MMA issuer, warp 2: TMA producer
-constexpr int kScoreStages = 6;
+constexpr int kScoreStages = 3;          // measured: 3-4 stages beat 6 (less queueing in the memory system)
 constexpr int kScoreTileBytes = 32768;
 constexpr int kScoreM = 64;               // MMA M: query heads of the group (<= 8), zero padded
 constexpr int kTmemCols = 512;
@@ -123,9 +123,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
     mbar_fence_init();
     *s_abort = 0;
   }
-  if (warp == 1) tmem_alloc(s_tmem, kTmemCols);
-  // everything below touches the workspace, which kernels of the previous call may still use
+  // everything below touches the workspace, which kernels of the previous call may still use;
+  // tensor memory is also taken only now, so that a CTA that started early never holds
+  // columns a CTA of a predecessor kernel is waiting for
   pdl_wait();
+  if (warp == 1) tmem_alloc(s_tmem, kTmemCols);
   // ---- clear this CTA's slice of the workspace head (counters, status word)
   {
     uint4* z = reinterpret_cast<uint4*>(p.status);
