@@ -181,6 +181,10 @@ tkphi_status tkphi_topk_decode(const tkphi_kv_desc* kv, const void* q,
  * subtraction, App. C.1) drops both residual terms, so y falls back to nu_E / Z_E.
  * With no anchor and no retrieved token the output is nu_hat_R / Z_hat_R; if that is
  * clamped as well the output row is zero.
+ * Generated tokens (Sec. 4.3, Eq. implemented_decode: tokens produced after the prefill
+ * stay in the exact branch): append their rows to the cache and pass n_tail + n_gen as the
+ * tail-anchor count of the decode call; the mid-region, and with it the meaning of (S, u)
+ * built at prefill time with n_tail, is unchanged.  All sequences of a call share n_gen.
  * Other arguments as for tkphi_topk_decode.
  */
 tkphi_status tkphi_decode_step(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, const void* q,

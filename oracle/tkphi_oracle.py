@@ -284,6 +284,48 @@ def topkphi_attention(q, K, V, n_sink, n_tail, topk, W_q, b_q, gamma_q, W_k, b_k
                                phi_log(q, W_q, b_q, gamma_q), Phi_ret, subtract=subtract)
 
 
+def topkphi_attention_generated(q, K_all, V_all, n_prefill: int, n_sink, n_tail, topk,
+                                W_q, b_q, gamma_q, W_k, b_k, gamma_k, S=None, u=None, retrieved=None):
+    """Decode with already generated tokens kept exact (Sec. 4.3, Eq. implemented_decode):
+
+        y_impl = (nu_E + nu_G + nu_hat_R) / (Z_E + Z_G + Z_hat_R).
+
+    K_all, V_all hold the n_prefill prefill rows followed by the generated rows G.  The
+    partition A, M, the selector and the summaries (S, u) refer to the prefill only; the
+    rows of G enter exactly, under the same normalisation.  Returns (y, retrieved).
+    """
+    K_all = np.asarray(K_all, F64)
+    V_all = np.asarray(V_all, F64)
+    L = int(n_prefill)
+    K, V = K_all[:L], V_all[:L]
+    if retrieved is None:
+        retrieved = select_topk(q, K, n_sink, n_tail, topk)
+    retrieved = np.asarray(retrieved, np.int64)
+    if S is None or u is None:
+        S, u = build_summaries(K, V, W_k, b_k, gamma_k, n_sink, n_tail)
+    E = exact_support(L, n_sink, n_tail, retrieved)
+    G = np.arange(L, K_all.shape[0], dtype=np.int64)
+    s_all = scores(q, K_all[np.concatenate([E, G])]) if E.size + G.size else np.zeros(0)
+    m_x = float(s_all.max()) if s_all.size else -math.inf
+    nu_E, Z_E = exact_terms(q, K_all, V_all, E, shift=m_x)
+    nu_G, Z_G = exact_terms(q, K_all, V_all, G, shift=m_x)
+    Phi_ret = (phi(K[retrieved], W_k, b_k, gamma_k) if retrieved.size
+               else np.zeros((0, np.asarray(W_k).shape[0]), F64))
+    S_R, u_R = subtract_retrieved(S, u, V, Phi_ret, retrieved)
+    a = phi_log(q, W_q, b_q, gamma_q)
+    m_q = float(a.max())
+    w = np.exp(a - m_q)
+    nu_t, Z_t = S_R @ w, float(w @ u_R)
+    if not (Z_t > 0.0):                      # clamp: residual dropped
+        return (nu_E + nu_G) / (Z_E + Z_G), retrieved
+    log_ZR = m_q + math.log(Z_t)
+    M = max(m_x, log_ZR)
+    cX = math.exp(m_x - M) if s_all.size else 0.0
+    cR = math.exp(log_ZR - M)
+    y = (cX * (nu_E + nu_G) + cR * (nu_t / Z_t)) / (cX * (Z_E + Z_G) + cR)
+    return y, retrieved
+
+
 def topkphi_reassociated(q, K, V, n_sink, n_tail, retrieved, S, u,
                          W_q, b_q, gamma_q, W_k, b_k, gamma_k):
     """Same output with the contraction reassociated:

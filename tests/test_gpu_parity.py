@@ -248,6 +248,34 @@ def test_exact_ties_break_towards_lower_index():
         _check_decode(gl2, 0, 0.0, None, None, with_phi=False, topk=[kk])
 
 
+def test_generated_tokens_stay_exact():
+    """Decode after n_gen generated tokens (Eq. implemented_decode): summaries from the prefill,
+    then a decode call whose tail-anchor count is n_tail + n_gen over the grown cache."""
+    import paper_2604_05438_b200 as T
+    cfg = _cfg("c1_1b_4k", n_q_heads=8, n_kv_heads=2)
+    L, n_gen = 2000, 37
+    inp = make_layer_inputs(cfg, 13, seq_lens=[L + n_gen], n_steps=1)
+    phi0 = make_phi_params(cfg, 13, kind="visible")
+    pre = dataclasses.replace(inp, cu_seqlens=np.array([0, L], np.int64), k=inp.k[:, :L].contiguous(),
+                              v=inp.v[:, :L].contiguous())
+    phi = make_phi_params(cfg, 13, kind="visible", bk_shift=PU.calibrate_visible_shift(cfg, pre, phi0, 0.02))
+    gl_pre = PU.to_gpu(cfg, pre, phi)
+    S, u = PU.gpu_build(gl_pre)                              # prefill state
+    grown = dataclasses.replace(inp, n_tail=cfg.n_tail + n_gen)
+    gl = PU.to_gpu(cfg, grown, phi)                          # cache with the generated rows appended
+    topk = np.array([39], np.int32)
+    out = PU.gpu_decode(gl, inp.q[0], topk, S, u)
+    Sh, uh = S.cpu().double().numpy(), u.cpu().double().numpy()
+    for hq in range(cfg.n_q_heads):
+        kvh = hq // cfg.group
+        K, V = PU.seq_arrays(inp, 0, kvh)
+        q64 = inp.q[0, 0, hq].double().numpy()
+        ret = PU.check_selection(q64, K[:L], cfg.n_sink, cfg.n_tail, 39, out["idx"][0, hq])
+        y0, _ = O.topkphi_attention_generated(q64, K, V, L, cfg.n_sink, cfg.n_tail, 39, *_phi_arrays(phi, hq, kvh),
+                                              S=Sh[0, kvh], u=uh[0, kvh], retrieved=ret)
+        assert PU.max_rel(out["y"][0, hq], y0) <= PU.Y_TOL, hq
+
+
 def test_results_are_run_to_run_identical():
     cfg = CONFIGS["c1_1b_4k"]
     inp = make_layer_inputs(cfg, 12, seq_lens=[2500], n_steps=1)

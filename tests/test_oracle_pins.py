@@ -358,3 +358,33 @@ def test_clamp_drops_nonpositive_residual():
     y_topk, _ = O.topk_attention(p["q"], p["K"], p["V"], 2, 3, 5)
     assert res.clamped and res.log_Zhat_R == -math.inf
     np.testing.assert_array_equal(res.y, y_topk)
+
+
+# ------------------------------------------------ generated tokens kept exact (Eq. implemented_decode)
+def test_generated_tokens_reduce_to_the_prefill_case_and_to_full_attention():
+    p = _rand_problem(41, L=60, d=8, r=6, n_sink=2, n_tail=5)
+    phi_args = (p["Wq"], p["bq"], 0.5, p["Wk"], p["bk"], 0.5)
+    # no generated token: the prefill-only estimator
+    y0, ret0 = O.topkphi_attention_generated(p["q"], p["K"], p["V"], 60, 2, 5, 9, *phi_args)
+    ref = O.topkphi_attention(p["q"], p["K"], p["V"], 2, 5, 9, *phi_args)
+    np.testing.assert_allclose(y0, ref.y, rtol=1e-12)
+    assert ret0.tolist() == ref.retrieved.tolist()
+    # 11 generated rows: the selector, the partition and (S, u) still see the 49 prefill rows only
+    L = 49
+    y1, ret1 = O.topkphi_attention_generated(p["q"], p["K"], p["V"], L, 2, 5, 9, *phi_args)
+    assert ret1.max() < L - 5 and ret1.tolist() == O.select_topk(p["q"], p["K"][:L], 2, 5, 9).tolist()
+    # with every mid token retrieved the residual vanishes and the result is full attention
+    # over prefill + generated rows
+    y2, _ = O.topkphi_attention_generated(p["q"], p["K"], p["V"], L, 2, 5, L - 7, *phi_args)
+    np.testing.assert_allclose(y2, O.full_attention(p["q"], p["K"], p["V"]), rtol=1e-9, atol=1e-12)
+    # the same numbers from the four terms of the equation written out one by one
+    ret = ret1
+    E = O.exact_support(L, 2, 5, ret)
+    G = np.arange(L, 60)
+    nu_E, Z_E = O.exact_terms(p["q"], p["K"], p["V"], E)
+    nu_G, Z_G = O.exact_terms(p["q"], p["K"], p["V"], G)
+    S, u = O.build_summaries(p["K"][:L], p["V"][:L], p["Wk"], p["bk"], 0.5, 2, 5)
+    S_R, u_R = O.subtract_retrieved(S, u, p["V"], O.phi(p["K"][ret], p["Wk"], p["bk"], 0.5), ret)
+    fq = O.phi(p["q"], p["Wq"], p["bq"], 0.5)
+    y_lit = (nu_E + nu_G + S_R @ fq) / (Z_E + Z_G + fq @ u_R)
+    np.testing.assert_allclose(y1, y_lit, rtol=1e-11)
