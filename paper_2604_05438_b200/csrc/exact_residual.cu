@@ -297,49 +297,78 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   // slice partials are combined in slice order by a fixed assignment of slices to
   // lanes and of output columns to threads, so the result does not depend on timing
   const float* parts = p.partials + (size_t)row * p.max_slices * p.partial_stride;
-  float m_loc = -INFINITY;
-  if (nE > 0)
-    for (int s = tid; s < n_slices; s += kExThreads) m_loc = fmaxf(m_loc, __ldcg(parts + (size_t)s * p.partial_stride));
-  m_loc = warp_max(m_loc);
-  if (lane == 0) misc[warp] = m_loc;
-  __syncthreads();
-  const float m_E = fmaxf(fmaxf(misc[0], misc[1]), fmaxf(misc[2], misc[3]));
-  if (warp == 0) {
-    float Zp = 0.f, zp = 0.f;
-    for (int s = lane; s < n_slices; s += 32) {
-      const float* ps = parts + (size_t)s * p.partial_stride;
-      const float f = nE > 0 ? expf(__ldcg(ps) - m_E) : 0.f;
-      Zp = fmaf(f, __ldcg(ps + 1), Zp);
-      zp += __ldcg(ps + 2);
+  constexpr int kFast = 16;                  // up to this many slices every load is issued at once
+  float m_E = -INFINITY, Z_E = 0.f, zs = 0.f, nu_E = 0.f, zv = 0.f;
+  const float* aqr = p.aq + (size_t)row * aq_stride(R, D);
+  float aq_m = 0.f, aq_u = 0.f, aq_s = 0.f;   // m_q, w . u_M, (S_M w)[tid]
+  if (p.with_phi) { aq_m = __ldcg(aqr + R); aq_u = __ldcg(aqr + R + 1); if (tid < D) aq_s = __ldcg(aqr + R + 4 + tid); }
+  if (n_slices <= kFast) {
+    // every thread combines the slice scalars itself (same order everywhere, no barrier)
+    float ms[kFast], Zs[kFast], zz[kFast], nus[kFast], zvs[kFast];
+    const int dv = tid < D ? tid : 0;
+#pragma unroll
+    for (int s = 0; s < kFast; ++s) {
+      const float* ps = parts + (size_t)(s < n_slices ? s : 0) * p.partial_stride;
+      ms[s] = __ldcg(ps); Zs[s] = __ldcg(ps + 1); zz[s] = __ldcg(ps + 2);
+      nus[s] = __ldcg(ps + 4 + dv); zvs[s] = __ldcg(ps + 4 + D + dv);
     }
-    Zp = warp_sum(Zp);
-    zp = warp_sum(zp);
-    if (lane == 0) { misc[4] = Zp; misc[5] = zp; }
-  }
-  float nu_E = 0.f, zv = 0.f;
-  if (tid < D) {
-#pragma unroll 4
-    for (int s = 0; s < n_slices; ++s) {
-      const float* ps = parts + (size_t)s * p.partial_stride;
-      const float f = nE > 0 ? expf(__ldcg(ps) - m_E) : 0.f;
-      nu_E = fmaf(f, __ldcg(ps + 4 + tid), nu_E);
-      zv += __ldcg(ps + 4 + D + tid);
+    if (nE > 0) {
+#pragma unroll
+      for (int s = 0; s < kFast; ++s) if (s < n_slices) m_E = fmaxf(m_E, ms[s]);
     }
+#pragma unroll
+    for (int s = 0; s < kFast; ++s) {
+      if (s < n_slices) {
+        const float f = nE > 0 ? expf(ms[s] - m_E) : 0.f;
+        Z_E = fmaf(f, Zs[s], Z_E);
+        zs += zz[s];
+        nu_E = fmaf(f, nus[s], nu_E);
+        zv += zvs[s];
+      }
+    }
+  } else {
+    float m_loc = -INFINITY;
+    if (nE > 0)
+      for (int s = tid; s < n_slices; s += kExThreads) m_loc = fmaxf(m_loc, __ldcg(parts + (size_t)s * p.partial_stride));
+    m_loc = warp_max(m_loc);
+    if (lane == 0) misc[warp] = m_loc;
+    __syncthreads();
+    m_E = fmaxf(fmaxf(misc[0], misc[1]), fmaxf(misc[2], misc[3]));
+    if (warp == 0) {
+      float Zp = 0.f, zp = 0.f;
+      for (int s = lane; s < n_slices; s += 32) {
+        const float* ps = parts + (size_t)s * p.partial_stride;
+        const float f = nE > 0 ? expf(__ldcg(ps) - m_E) : 0.f;
+        Zp = fmaf(f, __ldcg(ps + 1), Zp);
+        zp += __ldcg(ps + 2);
+      }
+      Zp = warp_sum(Zp);
+      zp = warp_sum(zp);
+      if (lane == 0) { misc[4] = Zp; misc[5] = zp; }
+    }
+    if (tid < D) {
+#pragma unroll 8
+      for (int s = 0; s < n_slices; ++s) {
+        const float* ps = parts + (size_t)s * p.partial_stride;
+        const float f = nE > 0 ? expf(__ldcg(ps) - m_E) : 0.f;
+        nu_E = fmaf(f, __ldcg(ps + 4 + tid), nu_E);
+        zv += __ldcg(ps + 4 + D + tid);
+      }
+    }
+    __syncthreads();
+    Z_E = misc[4]; zs = misc[5];
   }
-  __syncthreads();
-  const float Z_E = misc[4], zs = misc[5];
   float y = 0.f, yR = 0.f, logZR = -INFINITY, Mx = m_E;
   if (p.with_phi) {
     // S_M phi_q and phi_q . u_M (in units of exp(m_q)) were prepared alongside phi_q
-    const float* aqr = p.aq + (size_t)row * aq_stride(R, D);
-    const float m_q = aqr[R];
-    const float Zt = aqr[R + 1] - zs;                      // Z_hat_R / exp(m_q)
+    const float m_q = aq_m;
+    const float Zt = aq_u - zs;                            // Z_hat_R / exp(m_q)
     if (Zt > 0.f) {
       logZR = m_q + logf(Zt);
       Mx = fmaxf(m_E, logZR);
       const float cE = nE > 0 ? expf(m_E - Mx) : 0.f, cR = expf(logZR - Mx);
       if (tid < D) {
-        yR = (aqr[R + 4 + tid] - zv) / Zt;
+        yR = (aq_s - zv) / Zt;
         y = (cE * nu_E + cR * yR) / (cE * Z_E + cR);
       }
     } else if (tid < D) {

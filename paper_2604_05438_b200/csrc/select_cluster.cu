@@ -143,6 +143,7 @@ select_kernel(const Problem p, const int n_rows) {
   for (int i = tid; i < kHistBins; i += kSelThreads) { sm.hist[i] = 0; sm.acc[i] = 0; }
   for (int i = tid; i < kRefBins; i += kSelThreads) { sm.h1[i] = 0; sm.acc1[i] = 0; sm.acc2[i] = 0; }
   __syncthreads();
+  cluster.barrier_arrive();                                // "my accumulators are cleared"; waited for below
   for (int k = 0; k < rounds; ++k) {
     load_round(k);
 #pragma unroll 4
@@ -150,7 +151,7 @@ select_kernel(const Problem p, const int n_rows) {
       if ((vmask >> i) & 1u) atomicAdd(&sm.hist[keys[i * kSelThreads] >> kLowBits], 1u);
   }
   __syncthreads();
-  cluster.sync();                                          // every accumulator of the cluster is cleared
+  cluster.barrier_wait();                                  // every accumulator of the cluster is cleared
   push_all(sm.hist, sm.acc, kHistBins, false);
   cluster.sync();
   walk_from_top<kHistBins>(sm.acc, K, sm.res, sm.scratch);
