@@ -155,6 +155,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     // ================================================================ TMA producer
     if (lane == 0) {
       bool ok = true;
+      const uint64_t pol = l2_policy_evict_first();        // K and V are read once
       for (int it = 0; it < n_my && ok; ++it) {
         const int row = row0 + (t0 + it) * kBT;
         const int ks = it % KS, vs = it % VS;
@@ -163,7 +164,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
         mbar_expect_tx(&k_full[ks], C::TILE);
 #pragma unroll
         for (int x = 0; x < BOXES; ++x)
-          tma_load_3d(kring + ks * C::TILE + x * C::BOX, &tmap_k, &k_full[ks], x * 64, row, kvh);
+          tma_load_3d(kring + ks * C::TILE + x * C::BOX, &tmap_k, &k_full[ks], x * 64, row, kvh, pol);
         ok = mbar_wait(&v_empty[vs], ((uint32_t)(it / VS) & 1u) ^ 1u, s_abort);
         if (!ok) {
           // the key copy just issued must land before shared memory is released
@@ -176,7 +177,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
         mbar_expect_tx(&v_full[vs], C::TILE);
 #pragma unroll
         for (int x = 0; x < BOXES; ++x)
-          tma_load_3d(vring + vs * C::TILE + x * C::BOX, &tmap_v, &v_full[vs], x * 64, row, kvh);
+          tma_load_3d(vring + vs * C::TILE + x * C::BOX, &tmap_v, &v_full[vs], x * 64, row, kvh, pol);
       }
     }
   } else if (warp == 1) {

@@ -151,6 +151,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
         TileCursor pc;
         cursor_seek(pc, pre, batch, n_kv, f0);
         int it = 0, row_b = -1, row0 = 0;
+        const uint64_t pol = l2_policy_evict_first();      // the keys are read once
         for (; it < n_my; ++it) {
           const int slot = it % kScoreStages;
           const uint32_t ph = (uint32_t)(it / kScoreStages) & 1u;
@@ -161,7 +162,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
 #pragma unroll
           for (int x = 0; x < BOXES; ++x)
             tma_load_3d(tiles + slot * kScoreTileBytes + x * C::BOX_BYTES, &tmap_k, &full[slot], x * 64, row,
-                        pc.kvh);
+                        pc.kvh, pol);
           cursor_next(pc, pre, batch, n_kv);
         }
         if (it == n_my) {
