@@ -131,6 +131,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   // v into registers (its tile reuses the W_k region later).
   constexpr int CPR = D / 8;                 // 16-byte chunks per row = copies per thread
   uint4 vreg[CPR];
+  const uint64_t pol = l2_policy_evict_first();   // support rows are read once per head
 #pragma unroll
   for (int n = 0; n < CPR; ++n) {
     const int i = tid + n * kExThreads;
@@ -139,8 +140,8 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
     const uint32_t off = (c >> 3) * L::KV_BOX + swz128(t, c & 7);
     vreg[n] = make_uint4(0, 0, 0, 0);
     if (ti >= 0) {
-      vreg[n] = __ldg(reinterpret_cast<const uint4*>(vbase + (long long)ti * p.stride_token + c * 8));
-      if (!isret[t] || do_phi) cp_async_16(kt + off, kbase + (long long)ti * p.stride_token + c * 8);
+      vreg[n] = ld_global_16(vbase + (long long)ti * p.stride_token + c * 8, pol);
+      if (!isret[t] || do_phi) cp_async_16(kt + off, kbase + (long long)ti * p.stride_token + c * 8, pol);
       else *reinterpret_cast<uint4*>(kt + off) = make_uint4(0, 0, 0, 0);
     } else {
       *reinterpret_cast<uint4*>(kt + off) = make_uint4(0, 0, 0, 0);

@@ -243,6 +243,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
       long long len_b = 0;
       float* my_row = nullptr;
       const int g = lane >> 2, cpair = 2 * (lane & 3);
+      const uint64_t keep = l2_policy_evict_last();         // the score rows are read back right away
       bool ok = true;
       for (int it = 0; it < n_my && ok; ++it) {
         if (cc.b != cur_b || cc.kvh != cur_kvh) {
@@ -267,8 +268,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               const int j = j0 + half * 64 + i * 8;
-              if (j < n_mid) my_row[j] = v[4 * i] * p.scale;
-              if (j + 1 < n_mid) my_row[j + 1] = v[4 * i + 1] * p.scale;
+              if (j < n_mid) st_global_f32(my_row + j, v[4 * i] * p.scale, keep);
+              if (j + 1 < n_mid) st_global_f32(my_row + j + 1, v[4 * i + 1] * p.scale, keep);
             }
           }
         }
