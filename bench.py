@@ -104,15 +104,14 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- workload
-def algorithmic_bytes(cfg, n_tokens, topk, n_layers):
+def algorithmic_bytes(cfg, seq_lens, topk, n_layers):
     """Bytes the method itself must move per decode step (the score buffer is an
-    implementation artefact and is not counted)."""
+    implementation artefact and is not counted).  seq_lens, topk: per sequence."""
     d, r = cfg.head_dim, cfg.n_feat
     n_anchor = cfg.n_sink + cfg.n_tail
-    n_mid = n_tokens - n_anchor
-    key_stream = cfg.n_kv_heads * n_mid * d * 2
-    gather = cfg.n_q_heads * (topk + n_anchor) * 4 * d
-    su = cfg.n_kv_heads * (d * r + r) * 4
+    key_stream = sum(cfg.n_kv_heads * max(0, n - n_anchor) * d * 2 for n in seq_lens)
+    gather = sum(cfg.n_q_heads * (int(k) + min(n_anchor, n)) * 4 * d for n, k in zip(seq_lens, topk))
+    su = len(seq_lens) * cfg.n_kv_heads * (d * r + r) * 4
     weights = (cfg.n_q_heads + cfg.n_kv_heads) * (r * d + r) * 4
     per_layer = key_stream + gather + su + weights
     return {"key_stream": key_stream * n_layers, "total": per_layer * n_layers,
@@ -132,7 +131,8 @@ def run_ours(args, rank, world, device):
     layers, phis, Ss, us = [], [], [], []
     t_gen = time.time()
     for l in range(n_layers):
-        inp = make_layer_inputs(cfg, seed, layer=l, device=device, seq_lens=[N] * cfg.batch, n_steps=1)
+        inp = make_layer_inputs(cfg, seed, layer=l, device=device,
+                                seq_lens=([N] * cfg.batch) if (args.seq_len or cfg.seq_len_min is None) else None, n_steps=1)
         phi = make_phi_params(cfg, seed + l, device=device)
         kv = T.KVCache(inp.k, inp.v, inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, cfg.n_sink, cfg.n_tail)
         layers.append((inp, kv))
@@ -228,7 +228,8 @@ def run_ours(args, rank, world, device):
 
     ms, e2e_ms = max_over_ranks([total_ms / args.steps, e2e_ms], world, device)
 
-    ab = algorithmic_bytes(cfg, N, tmax, n_layers)
+    seq_lens = [layers[0][0].seq_len(b) for b in range(B)]
+    ab = algorithmic_bytes(cfg, seq_lens, topk, n_layers)
     peak, tf_burst, tf_sust, peak_kind = _peaks()
     out = {
         "metric": "Top-K+phi decode-step latency (us), 128K ctx",
@@ -236,7 +237,8 @@ def run_ours(args, rank, world, device):
         "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 K/V, f32 accumulate", "data": "synthetic",
         "config": {"workload": f"{cfg.name}: {n_layers} layers x {Hq}q/{Hkv}kv heads, d={d}, r={r}, N={N}, "
-                               f"anchors {cfg.n_sink}+{cfg.n_tail}, budget {args.budget:g} (K={tmax}), batch {B}",
+                               f"anchors {cfg.n_sink}+{cfg.n_tail}, budget {args.budget:g} (K<={tmax}), batch {B}"
+                               + (f", ragged lengths {min(seq_lens)}..{max(seq_lens)}" if len(set(seq_lens)) > 1 else ""),
                    "l2": "inputs (K/V of all layers) exceed L2 by >100x; no flush needed",
                    "replicas": world, "seed": seed},
         "step_us": {"median": statistics.median(per_step) * 1e3, "min": min(per_step) * 1e3,
@@ -248,7 +250,8 @@ def run_ours(args, rank, world, device):
         "gpu_launches": args.steps * n_layers * 3,
         "e2e": {"value": e2e_ms * 1e3, "unit": "us/step", "h2d_bytes_per_step": q_stage.numel() * 2,
                 "d2h_bytes_per_step": y_host.numel() * 4},
-        "build": build_info(build_ms, n_layers, B, Hkv, N - cfg.n_sink - cfg.n_tail, d, r, peak, tf_burst, tf_sust),
+        "build": build_info(build_ms, n_layers, Hkv, sum(max(0, n - cfg.n_sink - cfg.n_tail) for n in seq_lens), d, r,
+                            peak, tf_burst, tf_sust),
         "clocks": clocks,
         "gen_s": t_gen,
     }
@@ -278,11 +281,11 @@ def whole_job_steps_per_s(ms_per_step, world):
     return world * 1e3 / ms_per_step
 
 
-def build_info(build_ms, n_layers, B, Hkv, n_mid, d, r, hbm_peak, tf_burst, tf_sust):
+def build_info(build_ms, n_layers, Hkv, n_mid, d, r, hbm_peak, tf_burst, tf_sust):
     """Prefill summary build, timed separately: K and V of the mid-region are read once;
     the two contractions cost 2 * (2 n d r) flop per KV head, issued twice each (bf16 hi + lo)."""
-    kv_bytes = 2 * n_layers * B * Hkv * n_mid * d * 2
-    flops_alg = 4.0 * n_layers * B * Hkv * n_mid * d * r
+    kv_bytes = 2 * n_layers * Hkv * n_mid * d * 2          # n_mid: mid-region tokens summed over sequences
+    flops_alg = 4.0 * n_layers * Hkv * n_mid * d * r
     t = build_ms * 1e-3
     return {"ms_all_layers": build_ms, "kv_bytes": kv_bytes, "achieved_gbs": kv_bytes / t / 1e9,
             "hbm_frac_of_measured_peak": kv_bytes / t / 1e9 / hbm_peak,
