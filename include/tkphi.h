@@ -73,7 +73,8 @@ enum {
  * same strides.  Requirements: 1 <= batch <= 1024; head_dim in {64, 128}; n_q_heads a multiple of
  * n_kv_heads with group size <= 8; n_feat in {64, 128}; k and v 16-byte aligned;
  * both strides multiples of 8 elements; kv_stride_token >= head_dim; total rows
- * < 2^31.  Query head h_q uses KV head h_q / (n_q_heads / n_kv_heads).
+ * < 2^31; at most 2,097,152 mid-region rows per sequence for the decode entry points.
+ * Query head h_q uses KV head h_q / (n_q_heads / n_kv_heads).
  * Anchors (Eq. partition): the first n_sink and the last n_tail rows of each
  * sequence (their union when L_b < n_sink + n_tail); the mid-region is what lies
  * between, |M_b| = max(0, L_b - n_sink - n_tail).

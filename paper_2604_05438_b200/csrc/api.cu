@@ -58,7 +58,7 @@ tkphi_status validate_kv(const tkphi_kv_desc* kv, Shape* sh, bool need_data) {
   }
   sh->total_tokens = cu[kv->batch];
   sh->rows = kv->batch * kv->n_q_heads;
-  if ((long long)sh->rows + (sh->rows + kv->n_kv_heads + 7) / 8 > 65535)
+  if ((long long)sh->rows + sh->rows + kv->n_kv_heads > 65535)
     return fail(TKPHI_ERR_UNSUPPORTED, "batch * n_q_heads = %d is too large for one call", sh->rows);
   sh->units = kv->batch * kv->n_kv_heads;
   if (need_data) {
@@ -90,6 +90,8 @@ tkphi_status validate_topk(const tkphi_kv_desc* kv, const int32_t* topk_host, in
     if (!allow_empty_support && topk_host[b] == 0 && kv->n_sink == 0 && kv->n_tail == 0)
       return fail(TKPHI_ERR_INVALID_ARG, "sequence %d has an empty exact support (no anchors, topk = 0)", b);
     if (topk_host[b] > 0) sh->score_tiles += (int64_t)kv->n_kv_heads * ((mid + tk - 1) / tk);
+    if (mid > 2097152)
+      return fail(TKPHI_ERR_UNSUPPORTED, "sequence %d: mid-region of %lld tokens exceeds 2097152", b, (long long)mid);
   }
   if (sh->score_tiles >= (1ll << 31)) return fail(TKPHI_ERR_UNSUPPORTED, "too many key tiles");
   return TKPHI_OK;
@@ -283,7 +285,7 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   }
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_SELECT);
-    e = launch_select(p, cs);
+    e = launch_select(p, sh.score_tiles > 0 ? sh.max_mid : 0, cs);
   }
   if (e != cudaSuccess) return cuda_fail(e, "select launch");
   {

@@ -1,12 +1,13 @@
 // Exact Top-K selection over the score rows (exhaustive Top-K control selector, Sec. 5.1;
-// ties broken towards the lower index) in ONE kernel: a thread-block cluster of eight CTAs
-// per query head.
+// ties broken towards the lower index) in ONE kernel: a thread-block cluster of up to eight
+// CTAs per query head (1, 2, 4 or 8, enough to hold the longest row of the call).
 //
 // Each CTA owns a contiguous eighth of the head's mid-region; each warp a contiguous
 // 1024-score run of it, read coalesced (lane l, step i -> element 32 i + l), so that
 // (CTA, round, warp, step, lane) order is index order.  For sequences of up to 131072
 // mid-region keys every CTA keeps its 16384 order-preserving score keys in shared memory
-// and the row is read from L2 exactly once (the loops over a thread's 32 keys stay rolled:
+// and the row is read from L2 exactly once (longer rows, up to 2,097,152 keys, are read twice
+// and the shared memory holds per-round bit masks instead) (the loops over a thread's 32 keys stay rolled:
 // straight-line code that runs once is bound by instruction fetch, not by its work).  The exact K-th largest key is found by radix
 // selection over 12 + 10 + 10 bits: every CTA builds a local histogram in shared memory
 // and adds its non-zero bins into the accumulator of every CTA through distributed shared
@@ -32,7 +33,7 @@ namespace tkphi {
 constexpr int kSelThreads = 512;
 constexpr int kSelPer = 32;                              // scores per thread and round
 constexpr int kSelChunk = kSelThreads * kSelPer;         // 16384 scores per CTA and round
-constexpr int kSelCluster = 8;
+constexpr int kSelCluster = 8;                            // largest cluster; the launch picks 1, 2, 4 or 8
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kRefBins = 1024;                           // two refinement digits of 10 bits
 
@@ -73,8 +74,8 @@ __device__ void walk_from_top(const unsigned* h, int need, int* res, int* scratc
   __syncthreads();
 }
 
-__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads, 2)
-select_kernel(const Problem p, const int n_rows) {
+__global__ void __launch_bounds__(kSelThreads, 2)
+select_kernel(const Problem p, const int n_rows, const int csize) {
   __shared__ SelShared sm;
   extern __shared__ __align__(16) unsigned keys_s[];       // [kSelPer][kSelThreads]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -82,7 +83,7 @@ select_kernel(const Problem p, const int n_rows) {
   pdl_wait();                                              // score rows and workspace of the predecessors
   if ((int)blockIdx.y >= n_rows) {
     // ---- feature clusters: one task per CTA (query rows first, then KV heads)
-    const int task = ((int)blockIdx.y - n_rows) * kSelCluster + (int)blockIdx.x;
+    const int task = ((int)blockIdx.y - n_rows) * csize + (int)blockIdx.x;
     if (task < n_rows) {
       phi_q_stage1<kSelThreads>(p, task);
       __threadfence_block();
@@ -107,33 +108,39 @@ select_kernel(const Problem p, const int n_rows) {
   const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
   const float* srow = p.scores + score_row_base(p, b, hq, cu_b, len_b);
   const int n_chunks = (n_mid + kSelChunk - 1) / kSelChunk;
-  const int rounds = (n_chunks + kSelCluster - 1) / kSelCluster;      // per CTA
+  const int rounds = (n_chunks + csize - 1) / csize;       // per CTA
   const bool resident = rounds == 1;                       // the keys stay in shared memory
   const unsigned low_mask = (1u << kLowBits) - 1u;
 
-  // Order-preserving keys of this thread's 32 scores of round k go to shared memory
-  // (element i at keys[i * 512]); bit i of vmask <=> score i lies inside the row.
+  // Resident mode (one round per CTA): the order-preserving keys of this thread's 32 scores
+  // stay in shared memory (element i at keys[i * 512]) and its bit masks in registers.
+  // Otherwise (2..16 rounds) the keys are recomputed from the L2-resident row where needed and
+  // the shared-memory array holds the per-round bit masks instead.
   unsigned* keys = keys_s + tid;
-  unsigned vmask = 0;
-  auto load_round = [&](int k) {
-    const int base = (rank * rounds + k) * kSelChunk + warp * (32 * kSelPer) + lane;
+  const int base_w = warp * (32 * kSelPer) + lane;
+  auto round_base = [&](int k) { return (rank * rounds + k) * kSelChunk + base_w; };
+  auto load_regs = [&](int k, unsigned (&kr)[kSelPer]) -> unsigned {      // returns the validity mask
+    const int base = round_base(k);
     float sc[kSelPer];
 #pragma unroll
     for (int i = 0; i < kSelPer; ++i) sc[i] = (base + i * 32 < n_mid) ? __ldcg(srow + base + i * 32) : 0.f;
-    vmask = 0;
+    unsigned vm = 0;
 #pragma unroll
     for (int i = 0; i < kSelPer; ++i) {
-      keys[i * kSelThreads] = ordered_key(sc[i]);
-      if (base + i * 32 < n_mid) vmask |= 1u << i;
+      kr[i] = ordered_key(sc[i]);
+      if (base + i * 32 < n_mid) vm |= 1u << i;
     }
+    return vm;
+  };
+  auto key_at = [&](int k, int i) -> unsigned {            // key i of round k (valid positions only)
+    return resident ? keys[i * kSelThreads] : ordered_key(__ldcg(srow + round_base(k) + i * 32));
   };
   // adds the non-zero bins of a local histogram into the accumulator of every CTA
   auto push_all = [&](unsigned* local, unsigned* accum, int n_bins, bool clear) {
     for (int i = tid; i < n_bins; i += kSelThreads) {
       const unsigned c = local[i];
       if (c) {
-#pragma unroll
-        for (int r = 0; r < kSelCluster; ++r) atomicAdd(cluster.map_shared_rank(accum, r) + i, c);
+        for (int r = 0; r < csize; ++r) atomicAdd(cluster.map_shared_rank(accum, r) + i, c);
         if (clear) local[i] = 0;
       }
     }
@@ -144,11 +151,16 @@ select_kernel(const Problem p, const int n_rows) {
   for (int i = tid; i < kRefBins; i += kSelThreads) { sm.h1[i] = 0; sm.acc1[i] = 0; sm.acc2[i] = 0; }
   __syncthreads();
   cluster.barrier_arrive();                                // "my accumulators are cleared"; waited for below
+  unsigned vmask0 = 0;                                     // validity mask of the resident round
   for (int k = 0; k < rounds; ++k) {
-    load_round(k);
-#pragma unroll 4
-    for (int i = 0; i < kSelPer; ++i)
-      if ((vmask >> i) & 1u) atomicAdd(&sm.hist[keys[i * kSelThreads] >> kLowBits], 1u);
+    unsigned kr[kSelPer];
+    const unsigned vm = load_regs(k, kr);
+#pragma unroll
+    for (int i = 0; i < kSelPer; ++i) {
+      if (resident) keys[i * kSelThreads] = kr[i];
+      if ((vm >> i) & 1u) atomicAdd(&sm.hist[kr[i] >> kLowBits], 1u);
+    }
+    vmask0 = vm;
   }
   __syncthreads();
   cluster.barrier_wait();                                  // every accumulator of the cluster is cleared
@@ -160,30 +172,48 @@ select_kernel(const Problem p, const int n_rows) {
   const int n_cand = sm.res[2];
   const bool refine = need < n_cand;                       // the same in every CTA
 
-  // bit i of smask: key i lies above the threshold bin; of cmask: inside it
-  unsigned smask = 0, cmask = 0;
-  auto classify_round = [&]() {
-    smask = 0; cmask = 0;
+  // bit i of a "sure" mask: key i lies above the threshold bin; of a "cand" mask: inside it
+  unsigned smask = 0, cmask = 0;                           // resident mode
+  auto get_masks = [&](int k, unsigned* s_, unsigned* c_) {
+    if (resident) { *s_ = smask; *c_ = cmask; }
+    else { *s_ = keys_s[(2 * k) * kSelThreads + tid]; *c_ = keys_s[(2 * k + 1) * kSelThreads + tid]; }
+  };
+  auto put_masks = [&](int k, unsigned s_, unsigned c_) {
+    if (resident) { smask = s_; cmask = c_; }
+    else { keys_s[(2 * k) * kSelThreads + tid] = s_; keys_s[(2 * k + 1) * kSelThreads + tid] = c_; }
+  };
+  if (resident) {
+    unsigned s_ = 0, c_ = 0;
 #pragma unroll 4
     for (int i = 0; i < kSelPer; ++i) {
       const unsigned bin = keys[i * kSelThreads] >> kLowBits;
-      smask |= (bin > tb ? 1u : 0u) << i;
-      cmask |= (bin == tb ? 1u : 0u) << i;
+      s_ |= (bin > tb ? 1u : 0u) << i;
+      c_ |= (bin == tb ? 1u : 0u) << i;
     }
-    smask &= vmask; cmask &= vmask;
-  };
-  if (resident) classify_round();
+    smask = s_ & vmask0; cmask = c_ & vmask0;
+  } else {
+    for (int k = 0; k < rounds; ++k) {
+      unsigned kr[kSelPer];
+      const unsigned vm = load_regs(k, kr);
+      unsigned s_ = 0, c_ = 0;
+#pragma unroll
+      for (int i = 0; i < kSelPer; ++i) {
+        const unsigned bin = kr[i] >> kLowBits;
+        s_ |= (bin > tb ? 1u : 0u) << i;
+        c_ |= (bin == tb ? 1u : 0u) << i;
+      }
+      put_masks(k, s_ & vm, c_ & vm);
+    }
+  }
 
   unsigned tau_low = 0;
   int need_ties = n_cand;
   if (refine) {
     // ---- digit 1: bits 19..10 of the key among the keys of the threshold bin
     for (int k = 0; k < rounds; ++k) {
-      if (!resident) { load_round(k); classify_round(); }
-      for (unsigned m = cmask; m; m &= m - 1) {
-        const int i = __ffs(m) - 1;
-        atomicAdd(&sm.h1[(keys[i * kSelThreads] & low_mask) >> 10], 1u);
-      }
+      unsigned s_, c_;
+      get_masks(k, &s_, &c_);
+      for (unsigned m = c_; m; m &= m - 1) atomicAdd(&sm.h1[(key_at(k, __ffs(m) - 1) & low_mask) >> 10], 1u);
     }
     __syncthreads();
     push_all(sm.h1, sm.acc1, kRefBins, true);
@@ -194,10 +224,10 @@ select_kernel(const Problem p, const int n_rows) {
     __syncthreads();
     // ---- digit 2: bits 9..0 among the keys whose digit 1 matches
     for (int k = 0; k < rounds; ++k) {
-      if (!resident) { load_round(k); classify_round(); }
-      for (unsigned m = cmask; m; m &= m - 1) {
-        const int i = __ffs(m) - 1;
-        const unsigned low = keys[i * kSelThreads] & low_mask;
+      unsigned s_, c_;
+      get_masks(k, &s_, &c_);
+      for (unsigned m = c_; m; m &= m - 1) {
+        const unsigned low = key_at(k, __ffs(m) - 1) & low_mask;
         if ((low >> 10) == d1) atomicAdd(&sm.h1[low & (kRefBins - 1)], 1u);
       }
     }
@@ -209,34 +239,36 @@ select_kernel(const Problem p, const int n_rows) {
     need_ties = rem1 - sm.res[1];
   }
 
-  // after this, smask: keys above the exact threshold; cmask: keys equal to it (without
+  // after this, "sure": keys above the exact threshold; "cand": keys equal to it (without
   // refinement the whole threshold bin counts as tied: all of it is taken)
-  auto finish_masks = [&]() {
-    if (!refine) return;
-    unsigned tie = 0;
-    for (unsigned m = cmask; m; m &= m - 1) {
-      const int i = __ffs(m) - 1;
-      const unsigned low = keys[i * kSelThreads] & low_mask;
-      if (low > tau_low) smask |= 1u << i;
-      else if (low == tau_low) tie |= 1u << i;
+  if (refine) {
+    for (int k = 0; k < rounds; ++k) {
+      unsigned s_, c_, tie = 0;
+      get_masks(k, &s_, &c_);
+      for (unsigned m = c_; m; m &= m - 1) {
+        const int i = __ffs(m) - 1;
+        const unsigned low = key_at(k, i) & low_mask;
+        if (low > tau_low) s_ |= 1u << i;
+        else if (low == tau_low) tie |= 1u << i;
+      }
+      put_masks(k, s_, tie);
     }
-    cmask = tie;
-  };
-  if (resident) finish_masks();
+  }
 
   // ---- per-CTA totals, exchanged so that every CTA knows what the CTAs before it contribute
   {
     int n_sure = 0, n_tie = 0;
     for (int k = 0; k < rounds; ++k) {
-      if (!resident) { load_round(k); classify_round(); finish_masks(); }
-      n_sure += __popc(smask);
-      n_tie += __popc(cmask);
+      unsigned s_, c_;
+      get_masks(k, &s_, &c_);
+      n_sure += __popc(s_);
+      n_tie += __popc(c_);
     }
     n_sure = warp_sum_int(n_sure);
     n_tie = warp_sum_int(n_tie);
     if (lane == 0) { sm.wdef[warp] = n_sure; sm.wtie[warp] = n_tie; }
     __syncthreads();
-    if (tid < kSelCluster) {
+    if (tid < csize) {
       int a = 0, c = 0;
       for (int w = 0; w < kSelWarps; ++w) { a += sm.wdef[w]; c += sm.wtie[w]; }
       int* r = cluster.map_shared_rank(sm.tot, tid);
@@ -256,8 +288,9 @@ select_kernel(const Problem p, const int n_rows) {
 
   // ---- write the selected positions of this CTA in index order
   for (int k = 0; k < rounds; ++k) {
-    if (!resident) { load_round(k); classify_round(); finish_masks(); }
-    const int w_sure = warp_sum_int(__popc(smask)), w_tie = warp_sum_int(__popc(cmask));
+    unsigned smask_k, cmask_k;
+    get_masks(k, &smask_k, &cmask_k);
+    const int w_sure = warp_sum_int(__popc(smask_k)), w_tie = warp_sum_int(__popc(cmask_k));
     __syncthreads();                                       // wdef / wtie of the previous use are read
     if (lane == 0) { sm.wdef[warp] = w_sure; sm.wtie[warp] = w_tie; }
     __syncthreads();
@@ -272,12 +305,12 @@ select_kernel(const Problem p, const int n_rows) {
       r_sel += sm.wdef[w] + take;
     }
     const unsigned lt = (1u << lane) - 1u;
-    const int pos0 = p.n_sink + (rank * rounds + k) * kSelChunk + warp * (32 * kSelPer) + lane;
+    const int pos0 = p.n_sink + round_base(k);
     if (w_sure + w_tie > 0) {                              // most warps of most rounds hold nothing
 #pragma unroll 2
       for (int i = 0; i < kSelPer; ++i) {
-        const bool t = (cmask >> i) & 1u;
-        const unsigned sure_m = __ballot_sync(0xffffffffu, (smask >> i) & 1u);
+        const bool t = (cmask_k >> i) & 1u;
+        const unsigned sure_m = __ballot_sync(0xffffffffu, (smask_k >> i) & 1u);
         const unsigned tie_m = __ballot_sync(0xffffffffu, t);
         if ((sure_m | tie_m) == 0) continue;
         int n_take = need_ties - tie_run;                  // ties of this step that are still admitted
@@ -301,11 +334,13 @@ select_kernel(const Problem p, const int n_rows) {
   }
 }
 
-cudaError_t launch_select(const Problem& p, cudaStream_t st) {
+cudaError_t launch_select(const Problem& p, int max_mid, cudaStream_t st) {
   const int rows = p.batch * p.n_q_heads;
+  // cluster size: enough CTAs to keep the longest row in shared memory, at most 8
+  int csize = 1;
+  while (csize < kSelCluster && (long long)csize * kSelChunk < max_mid) csize *= 2;
   const int n_tasks = p.with_phi ? rows + p.n_kv_heads : 0;
-  const int feat_clusters = (n_tasks + kSelCluster - 1) / kSelCluster;
-  dim3 grid(kSelCluster, rows + feat_clusters, 1);
+  const int feat_clusters = (n_tasks + csize - 1) / csize;
   static bool configured = false;
   constexpr size_t smem = sizeof(unsigned) * kSelChunk;
   if (!configured) {
@@ -313,7 +348,18 @@ cudaError_t launch_select(const Problem& p, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  return launch_pdl(select_kernel, grid, dim3(kSelThreads), smem, st, p, rows);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(csize, rows + feat_clusters, 1);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = csize; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, select_kernel, p, rows, csize);
 }
 
 }  // namespace tkphi
