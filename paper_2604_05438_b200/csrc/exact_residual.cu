@@ -13,7 +13,9 @@
 // retrieved token contribute to both branches while its v row is in shared memory.
 // phi_q is carried as exp(a_q - m_q) with the log-scale m_q separate.
 //
-// The support list of a query head is cut into slices of 128 tokens, one CTA each.
+// The support list of a query head is cut into slices of 128 tokens; a CTA takes two
+// adjacent slices, one per group of 128 threads, which share the W_k operand tiles (so a
+// decode call at a 1% budget of a 128K context is a single wave of one CTA per SM).
 // The k and v rows of a slice are gathered into 128B-swizzled shared-memory tiles.
 // The feature recompute of the retrieved keys, W_k k_i for 128 tokens x r features, is
 // a dense [128 x d] x [d x r] contraction: it runs as tcgen05.mma with the gathered key
@@ -28,48 +30,51 @@
 
 namespace tkphi {
 
-constexpr int kExThreads = 128;      // one thread per token of the slice = per tensor-memory lane
+constexpr int kExGroups = 2;                        // slices per CTA
+constexpr int kExThreads = kExGroups * kSlice;      // one thread per token of a slice = per tensor-memory lane
 
 template <int D, int R>
 struct ExSmem {
   static constexpr int BOXES = D / 64;
   static constexpr int KV_BOX = kSlice * 128;                 // bytes of one 64-dim column block of k or v
   static constexpr int W_BOX = R * 128;
-  static constexpr size_t kt = 0;                             // bf16 k tile  [BOXES][128][128 B]
-  static constexpr size_t whi = kt + (size_t)BOXES * KV_BOX;  // bf16 W_k hi  [BOXES][R][128 B]
+  static constexpr size_t kv_tile = (size_t)BOXES * KV_BOX;   // one k or v tile [BOXES][128][128 B]
+  static constexpr size_t kt = 0;                             // bf16 k tiles, one per group
+  static constexpr size_t whi = kt + kExGroups * kv_tile;     // bf16 W_k hi  [BOXES][R][128 B]
   static constexpr size_t wlo = whi + (size_t)BOXES * W_BOX;
-  // the v tile takes over the W_k region once the MMAs have read it (the v rows wait in
-  // registers until then), which keeps the CTA small enough for two per SM
+  // the v tiles take over the W_k region once the MMAs have read it (the v rows wait in
+  // registers until then)
   static constexpr size_t vt = whi;
-  static constexpr size_t w_bytes = 2 * (size_t)BOXES * W_BOX, v_bytes = (size_t)BOXES * KV_BOX;
+  static constexpr size_t w_bytes = 2 * (size_t)BOXES * W_BOX, v_bytes = kExGroups * kv_tile;
   static constexpr size_t small = whi + (w_bytes > v_bytes ? w_bytes : v_bytes);
-  // small: bars[2] (16 B), tok[128] int, isret[128] int, wgt[128], zt[128], qf[D], cj[R], spare[R],
-  //        red[4*D], misc[16]
-  static constexpr size_t total = small + 16 + 4 * (4 * kSlice + D + 2 * R + 4 * D + 16);
+  // small: bars[4] (32 B), tok[T] int, isret[T] int, wgt[T], zt[T] (T threads), qf[D], cj[R], spare[R],
+  //        red[groups][4*D], misc[32]
+  static constexpr size_t total = small + 32 + 4 * (4 * kExThreads + D + 2 * R + kExGroups * 4 * D + 32);
 };
 
 template <int D, int R>
 __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Problem p) {
   using L = ExSmem<D, R>;
   extern __shared__ __align__(1024) unsigned char smem[];
-  unsigned char* kt = smem + L::kt;
-  unsigned char* vt = smem + L::vt;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int grp = tid / kSlice, gt = tid % kSlice, gwarp = warp & 3;   // group, token (= tensor-memory lane), warp of the group
+  unsigned char* kt = smem + L::kt + grp * L::kv_tile;      // this group's tiles
+  unsigned char* vt = smem + L::vt + grp * L::kv_tile;
   unsigned char* whi = smem + L::whi;
   unsigned char* wlo = smem + L::wlo;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::small);   // [0]: W tiles landed, [1]: MMAs done
-  int* tok = reinterpret_cast<int*>(bars + 2);
-  int* isret = tok + kSlice;
-  float* wgt = reinterpret_cast<float*>(isret + kSlice);
-  float* zt = wgt + kSlice;
-  float* qf = zt + kSlice;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::small);   // [0]: W tiles landed, [1 + g]: MMAs of group g done
+  int* tok = reinterpret_cast<int*>(bars + 4) + grp * kSlice;        // per-token arrays: this group's part
+  int* isret = reinterpret_cast<int*>(bars + 4) + kExThreads + grp * kSlice;
+  float* wgt = reinterpret_cast<float*>(bars + 4) + 2 * kExThreads + grp * kSlice;
+  float* zt = reinterpret_cast<float*>(bars + 4) + 3 * kExThreads + grp * kSlice;
+  float* qf = reinterpret_cast<float*>(bars + 4) + 4 * kExThreads;
   float* cj = qf + D;               // log2 w_j + b_k[j] log2 e
-  float* red = cj + 2 * R;
-  float* misc = red + 4 * D;
-  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 12);
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 13);
+  float* red = cj + 2 * R + grp * 4 * D;
+  float* misc = cj + 2 * R + kExGroups * 4 * D;
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 28);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 29);
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = blockIdx.z, hq = blockIdx.y, slice = blockIdx.x;
+  const int b = blockIdx.z, hq = blockIdx.y, slice0 = blockIdx.x * kExGroups, slice = slice0 + grp;
   pdl_launch_next();
   const int row = b * p.n_q_heads + hq, kvh = hq / p.group;
   const int K = p.topk[b];
@@ -81,10 +86,16 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   const int tail_start = (int)ts, n_tail_eff = (int)(len_b - ts);
   const int nE = nA1 + K + n_tail_eff;
   const int n_slices = nE > 0 ? (nE + kSlice - 1) / kSlice : 1;
-  if (slice >= n_slices) return;
+  if (slice0 >= n_slices) return;
+  const int n_ctas = (n_slices + kExGroups - 1) / kExGroups;
+  const bool live = slice < n_slices;            // the last CTA of a head may hold one empty group
   const bool do_phi = p.with_phi && !(p.flags & 1u);
-  // does this slice hold retrieved tokens (positions nA1 .. nA1+K-1 of the support list)?
-  const bool has_ret = do_phi && slice * kSlice < nA1 + K && (slice + 1) * kSlice > nA1;
+  // does a slice hold retrieved tokens (positions nA1 .. nA1+K-1 of the support list)?
+  auto slice_has_ret = [&](int s) { return do_phi && s < n_slices && s * kSlice < nA1 + K && (s + 1) * kSlice > nA1; };
+  const bool has_ret = slice_has_ret(slice);
+  bool any_ret = false;
+#pragma unroll
+  for (int g = 0; g < kExGroups; ++g) any_ret = any_ret || slice_has_ret(slice0 + g);
 
   const __nv_bfloat16* kbase = p.k + (long long)kvh * p.stride_head + cu_b * p.stride_token;
   const __nv_bfloat16* vbase = p.v + (long long)kvh * p.stride_head + cu_b * p.stride_token;
@@ -93,23 +104,24 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   // ---- 0. barriers, tensor memory, W_k operand tiles
   if (tid == 0) {
     mbar_init(&bars[0], 1);
-    mbar_init(&bars[1], 1);
+#pragma unroll
+    for (int g = 0; g < kExGroups; ++g) mbar_init(&bars[1 + g], 1);
     mbar_fence_init();
     *s_abort = 0;
   }
   pdl_wait();                                  // the index lists, features and score rows of the predecessors
-  if (has_ret && warp == 0) tmem_alloc(s_tmem, R);   // after the wait: never hold columns a predecessor needs
+  if (any_ret && warp == 0) tmem_alloc(s_tmem, kExGroups * R);   // after the wait: never hold columns a predecessor needs
   // ---- 1. token list of this slice
   {
-    const int pi = slice * kSlice + tid;
+    const int pi = slice * kSlice + gt;
     int t = -1, ret = 0;
-    if (pi < nE) {
+    if (live && pi < nE) {
       if (pi < nA1) t = pi;
       else if (pi < nA1 + K) { t = p.idx[(size_t)row * p.topk_max + (pi - nA1)]; ret = 1; }
       else t = tail_start + (pi - nA1 - K);
     }
-    tok[tid] = t;
-    isret[tid] = ret;
+    tok[gt] = t;
+    isret[gt] = ret;
   }
   for (int c = tid; c < D; c += kExThreads) qf[c] = __bfloat162float(p.q[(size_t)row * D + c]);
   if (do_phi) {
@@ -119,7 +131,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  if (has_ret && tid == 0) {
+  if (any_ret && tid == 0) {
     const unsigned char* img = reinterpret_cast<const unsigned char*>(p.wk_img + (size_t)kvh * 2 * R * D);
     mbar_expect_tx(&bars[0], 2u * R * D * 2u);
     bulk_load(whi, img, R * D * 2, &bars[0]);
@@ -134,7 +146,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   const uint64_t pol = l2_policy_evict_first();   // support rows are read once per head
 #pragma unroll
   for (int n = 0; n < CPR; ++n) {
-    const int i = tid + n * kExThreads;
+    const int i = gt + n * kSlice;
     const int t = i / CPR, c = i % CPR;
     const int ti = tok[t];
     const uint32_t off = (c >> 3) * L::KV_BOX + swz128(t, c & 7);
@@ -153,33 +165,37 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
 
   // ---- 3. feature recompute on the tensor core: acc[t][j] = sum_c k_t[c] (W_hi + W_lo)[j][c]
   bool ok = true;
-  if (has_ret && tid == 0) {
+  if (any_ret && tid == 0) {
     ok = mbar_wait(&bars[0], 0, s_abort);
     if (ok) {
       tc_fence_after_sync();
       constexpr uint32_t idesc = umma_idesc_bf16(128, R, 0, 0);
-      const uint32_t tmem_d = *s_tmem;
-      const uint64_t adesc0 = umma_smem_desc(smem_u32(kt), 16, 1024);
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint64_t bdesc0 = umma_smem_desc(smem_u32(half == 0 ? whi : wlo), 16, 1024);
+      for (int g = 0; g < kExGroups; ++g) {
+        if (!slice_has_ret(slice0 + g)) continue;
+        const uint32_t tmem_d = *s_tmem + g * R;             // group g accumulates in columns [g R, (g+1) R)
+        const uint64_t adesc0 = umma_smem_desc(smem_u32(smem + L::kt + g * L::kv_tile), 16, 1024);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          umma_ss(tmem_d, adesc0 + (uint64_t)(((k >> 2) * L::KV_BOX + (k & 3) * 32) >> 4),
-                  bdesc0 + (uint64_t)(((k >> 2) * L::W_BOX + (k & 3) * 32) >> 4), idesc, (half | k) ? 1u : 0u);
+        for (int half = 0; half < 2; ++half) {
+          const uint64_t bdesc0 = umma_smem_desc(smem_u32(half == 0 ? whi : wlo), 16, 1024);
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k)
+            umma_ss(tmem_d, adesc0 + (uint64_t)(((k >> 2) * L::KV_BOX + (k & 3) * 32) >> 4),
+                    bdesc0 + (uint64_t)(((k >> 2) * L::W_BOX + (k & 3) * 32) >> 4), idesc, (half | k) ? 1u : 0u);
+        }
+        tc_commit(&bars[1 + g]);
       }
-      tc_commit(&bars[1]);
     }
   }
 
   // ---- 4. per token (thread = token): |k|^2, anchor score, softmax weight
-  const int ti = tok[tid];
+  const int ti = tok[gt];
   float s_val = -INFINITY, kn = 0.f;
   if (ti >= 0) {
     float dot = 0.f;
 #pragma unroll
     for (int c = 0; c < CPR; ++c) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(kt + (c >> 3) * L::KV_BOX + swz128(tid, c & 7));
+      const uint4 raw = *reinterpret_cast<const uint4*>(kt + (c >> 3) * L::KV_BOX + swz128(gt, c & 7));
       const unsigned w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -190,54 +206,52 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
         kn = fmaf(x1, x1, kn);
       }
     }
-    s_val = isret[tid] ? srow[ti - p.n_sink] : dot * p.scale;
+    s_val = isret[gt] ? srow[ti - p.n_sink] : dot * p.scale;
   }
   {
     const float m = warp_max(s_val);
     if (lane == 0) misc[warp] = m;
   }
   __syncthreads();
-  const float m_slice = fmaxf(fmaxf(misc[0], misc[1]), fmaxf(misc[2], misc[3]));
+  const float m_slice = fmaxf(fmaxf(misc[4 * grp], misc[4 * grp + 1]), fmaxf(misc[4 * grp + 2], misc[4 * grp + 3]));
   const float w_t = ti >= 0 ? expf(s_val - m_slice) : 0.f;
-  wgt[tid] = w_t;
+  wgt[gt] = w_t;
 
   // ---- 5. z_t = <phi_q, phi_k(k_t)> from the accumulator row of this token
   float z_t = 0.f;
-  if (has_ret) {
-    ok = mbar_wait(&bars[1], 0, s_abort);
-    ok = __syncthreads_and(ok ? 1 : 0) != 0;       // the MMAs are done: W_k tiles are free
-  }
+  if (has_ret) ok = mbar_wait(&bars[1 + grp], 0, s_abort);
+  ok = __syncthreads_and(ok ? 1 : 0) != 0;         // every group's MMAs are done: the W_k tiles are free
   // the v rows move from registers into their tile (over the W_k region)
 #pragma unroll
   for (int n = 0; n < CPR; ++n) {
-    const int i = tid + n * kExThreads;
+    const int i = gt + n * kSlice;
     const int t = i / CPR, c = i % CPR;
     *reinterpret_cast<uint4*>(vt + (c >> 3) * L::KV_BOX + swz128(t, c & 7)) = vreg[n];
   }
   if (has_ret && ok) {
     tc_fence_after_sync();
-    const uint32_t tmem_d = *s_tmem;
+    const uint32_t tmem_d = *s_tmem + grp * R;
     // z = 2^(-gamma log2e |k|^2) * sum_j 2^(acc_j + c_j): four partial sums in a fixed order
     float zp[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int c4 = 0; c4 < R / 32; ++c4) {
       float v[32];
-      tmem_ld_x32(tmem_addr(tmem_d, warp * 32, c4 * 32), v);
+      tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, c4 * 32), v);
       tc_wait_ld();
 #pragma unroll
       for (int j = 0; j < 32; ++j) zp[j & 3] += ex2_approx(v[j] + cj[c4 * 32 + j]);
     }
     z_t = ((zp[0] + zp[1]) + (zp[2] + zp[3])) * ex2_approx(-p.gamma_k * kLog2e * kn);
-    if (!isret[tid]) z_t = 0.f;
+    if (!isret[gt]) z_t = 0.f;
   }
-  zt[tid] = z_t;
+  zt[gt] = z_t;
   __syncthreads();
 
   // ---- 6. slice partials: nu = sum w_t v_t, zv = sum z_t v_t, Z = sum w_t, zs = sum z_t
   {
-    constexpr int NGV = kExThreads / D;      // token groups for the value pass (1 or 2)
+    constexpr int NGV = kSlice / D;          // token groups for the value pass (1 or 2)
     constexpr int TPV = kSlice / NGV;
-    const int dv = tid % D, tg = tid / D;
+    const int dv = gt % D, tg = gt / D;
     const unsigned char* vcol = vt + (dv >> 6) * L::KV_BOX + (dv & 7) * 2;
     const uint32_t ch = (dv & 63) >> 3;
     float nu0 = 0.f, nu1 = 0.f, zv0 = 0.f, zv1 = 0.f;      // even / odd tokens, added in a fixed order
@@ -257,39 +271,41 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   }
   __syncthreads();
   float* part = p.partials + ((size_t)row * p.max_slices + slice) * p.partial_stride;
-  for (int i = tid; i < 2 * D; i += kExThreads) {
-    constexpr int NGV = kExThreads / D;
-    float x = red[i];
-    if (NGV == 2) x += red[2 * D + i];       // second token group, fixed order
-    part[4 + i] = x;
-  }
-  if (tid < 32) {
-    float Z = 0.f, zs = 0.f;
+  if (live) {
+    for (int i = gt; i < 2 * D; i += kSlice) {
+      constexpr int NGV = kSlice / D;
+      float x = red[i];
+      if (NGV == 2) x += red[2 * D + i];     // second token group, fixed order
+      part[4 + i] = x;
+    }
+    if (gwarp == 0) {
+      float Z = 0.f, zs = 0.f;
 #pragma unroll
-    for (int i = 0; i < kSlice / 32; ++i) { Z += wgt[tid + 32 * i]; zs += zt[tid + 32 * i]; }
-    Z = warp_sum(Z);
-    zs = warp_sum(zs);
-    if (tid == 0) { part[0] = m_slice; part[1] = Z; part[2] = zs; part[3] = 0.f; }
+      for (int i = 0; i < kSlice / 32; ++i) { Z += wgt[lane + 32 * i]; zs += zt[lane + 32 * i]; }
+      Z = warp_sum(Z);
+      zs = warp_sum(zs);
+      if (lane == 0) { part[0] = m_slice; part[1] = Z; part[2] = zs; part[3] = 0.f; }
+    }
   }
 
   // ---- tensor memory is no longer needed
   tc_fence_before_sync();
   __syncthreads();
-  if (has_ret && warp == 0) {
+  if (any_ret && warp == 0) {
     tc_fence_after_sync();
-    tmem_dealloc(*s_tmem, R);
+    tmem_dealloc(*s_tmem, kExGroups * R);
   }
   if (*s_abort) {
     if (tid == 0) atomicExch(p.status, kStatusTimeout);
     return;
   }
 
-  // ---- ticket: the last slice CTA of this head merges
+  // ---- ticket: the last CTA of this head merges
   __threadfence();
   __syncthreads();
   if (tid == 0) {
     const unsigned prev = atomicAdd(&p.row_counter[row], 1u);
-    misc[8] = (prev == (unsigned)(n_slices - 1)) ? 1.f : 0.f;
+    misc[8] = (prev == (unsigned)(n_ctas - 1)) ? 1.f : 0.f;
   }
   __syncthreads();
   if (misc[8] == 0.f) return;
@@ -334,7 +350,8 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
     m_loc = warp_max(m_loc);
     if (lane == 0) misc[warp] = m_loc;
     __syncthreads();
-    m_E = fmaxf(fmaxf(misc[0], misc[1]), fmaxf(misc[2], misc[3]));
+#pragma unroll
+    for (int w = 0; w < kExThreads / 32; ++w) m_E = fmaxf(m_E, misc[w]);
     if (warp == 0) {
       float Zp = 0.f, zp = 0.f;
       for (int s = lane; s < n_slices; s += 32) {
@@ -345,7 +362,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
       }
       Zp = warp_sum(Zp);
       zp = warp_sum(zp);
-      if (lane == 0) { misc[4] = Zp; misc[5] = zp; }
+      if (lane == 0) { misc[16] = Zp; misc[17] = zp; }
     }
     if (tid < D) {
 #pragma unroll 8
@@ -357,7 +374,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
       }
     }
     __syncthreads();
-    Z_E = misc[4]; zs = misc[5];
+    Z_E = misc[16]; zs = misc[17];
   }
   float y = 0.f, yR = 0.f, logZR = -INFINITY, Mx = m_E;
   if (p.with_phi) {
@@ -396,7 +413,7 @@ static cudaError_t launch_ex_t(const Problem& p, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid(p.max_slices, p.n_q_heads, p.batch);
+  dim3 grid((p.max_slices + kExGroups - 1) / kExGroups, p.n_q_heads, p.batch);
   return launch_pdl(exact_residual_kernel<D, R>, grid, dim3(kExThreads), smem, st, p);
 }
 
