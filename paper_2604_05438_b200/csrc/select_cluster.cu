@@ -13,9 +13,9 @@
 // and adds its non-zero bins into the accumulator of every CTA through distributed shared
 // memory; every CTA then walks its own copy of the accumulator.  Positions above the
 // threshold, and as many threshold ties as are still needed in index order, are then
-// written straight to their slot of the ascending index list: offsets come from warp
-// ballots, a scan over the warps of a CTA, and per-CTA totals exchanged through
-// distributed shared memory.  CTAs of a cluster only meet at hardware cluster barriers
+// written straight to their slot of the ascending index list: the per-thread bit masks
+// are transposed inside each warp so that thread order is index order, and offsets come
+// from one block scan and per-CTA totals exchanged through distributed shared memory.  CTAs of a cluster only meet at hardware cluster barriers
 // (no flag spinning, no global scratch, nothing to clear between calls).
 //
 // Extra clusters of the same launch do the work that depends only on the call's inputs
@@ -72,6 +72,20 @@ __device__ void walk_from_top(const unsigned* h, int need, int* res, int* scratc
     }
   }
   __syncthreads();
+}
+
+// Transposes the 32 x 32 bit matrix whose row l is the word of lane l: afterwards bit j of
+// lane t is what bit t of lane j was.
+__device__ __forceinline__ unsigned warp_transpose32(unsigned x, int lane) {
+  unsigned m = 0x0000ffffu;
+#pragma unroll
+  for (int j = 16; j; j >>= 1) {
+    const unsigned y = __shfl_xor_sync(0xffffffffu, x, j);
+    if ((lane & j) == 0) x ^= (((x >> j) ^ y) & m) << j;
+    else x ^= ((y >> j) ^ x) & m;
+    m ^= m << (j >> 1);
+  }
+  return x;
 }
 
 __global__ void __launch_bounds__(kSelThreads, 2)
@@ -286,51 +300,37 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
     tie_base += t;
   }
 
-  // ---- write the selected positions of this CTA in index order
+  // ---- write the selected positions of this CTA in index order.  The masks are transposed
+  // inside each warp first, so that lane t holds the bits of the 32 consecutive positions
+  // 32 t .. 32 t + 31 of the warp's run and thread order is index order; one block scan of
+  // the packed (tie, sure) counts then gives every thread its first output slot.
   for (int k = 0; k < rounds; ++k) {
-    unsigned smask_k, cmask_k;
-    get_masks(k, &smask_k, &cmask_k);
-    const int w_sure = warp_sum_int(__popc(smask_k)), w_tie = warp_sum_int(__popc(cmask_k));
-    __syncthreads();                                       // wdef / wtie of the previous use are read
-    if (lane == 0) { sm.wdef[warp] = w_sure; sm.wtie[warp] = w_tie; }
-    __syncthreads();
-    int tie_run = tie_base, out_run = out_base;            // before this warp, then before this step
-    int r_tie = 0, r_sel = 0;                              // this round's totals
-    for (int w = 0; w < kSelWarps; ++w) {
-      const int t = sm.wtie[w];
-      int take = need_ties - (tie_base + r_tie);
-      take = take < 0 ? 0 : (take > t ? t : take);
-      if (w < warp) { tie_run += t; out_run += sm.wdef[w] + take; }
-      r_tie += t;
-      r_sel += sm.wdef[w] + take;
-    }
-    const unsigned lt = (1u << lane) - 1u;
-    const int pos0 = p.n_sink + round_base(k);
-    if (w_sure + w_tie > 0) {                              // most warps of most rounds hold nothing
-#pragma unroll 2
-      for (int i = 0; i < kSelPer; ++i) {
-        const bool t = (cmask_k >> i) & 1u;
-        const unsigned sure_m = __ballot_sync(0xffffffffu, (smask_k >> i) & 1u);
-        const unsigned tie_m = __ballot_sync(0xffffffffu, t);
-        if ((sure_m | tie_m) == 0) continue;
-        int n_take = need_ties - tie_run;                  // ties of this step that are still admitted
-        const int nt = __popc(tie_m);
-        n_take = n_take < 0 ? 0 : (n_take > nt ? nt : n_take);
-        const bool taken = t && __popc(tie_m & lt) < n_take;
-        const unsigned sel = sure_m | __ballot_sync(0xffffffffu, taken);
-        if ((sel >> lane) & 1u) {
-          const int off = out_run + __popc(sel & lt);
-          if (off < K) {
-            out[off] = pos0 + i * 32;
-            if (out2) out2[off] = pos0 + i * 32;
-          }
+    unsigned s_, c_;
+    get_masks(k, &s_, &c_);
+    s_ = warp_transpose32(s_, lane);
+    c_ = warp_transpose32(c_, lane);
+    const int nt = __popc(c_);
+    int total;
+    const int excl = block_exclusive_scan((nt << 16) | __popc(s_), sm.scratch, &total);   // counts <= 16384 each
+    const int admit = max(need_ties - tie_base, 0);        // ties of this round that are still admitted
+    const int ties_before = excl >> 16;
+    int off = out_base + (excl & 0xffff) + min(ties_before, admit);
+    int take = min(max(admit - ties_before, 0), nt);       // admitted ties of this thread, in index order
+    const int pos0 = p.n_sink + (rank * rounds + k) * kSelChunk + warp * (32 * kSelPer) + lane * kSelPer;
+    for (unsigned m = s_ | c_; m; m &= m - 1) {
+      const int i = __ffs(m) - 1;
+      bool sel = (s_ >> i) & 1u;
+      if (!sel) { sel = take > 0; --take; }
+      if (sel) {
+        if (off < K) {
+          out[off] = pos0 + i;
+          if (out2) out2[off] = pos0 + i;
         }
-        out_run += __popc(sel);
-        tie_run += nt;
+        ++off;
       }
     }
-    tie_base += r_tie;
-    out_base += r_sel;
+    out_base += (total & 0xffff) + min(total >> 16, admit);
+    tie_base += total >> 16;
   }
 }
 
