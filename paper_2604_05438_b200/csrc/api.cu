@@ -285,7 +285,7 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   }
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_SELECT);
-    e = launch_select(p, sh.score_tiles > 0 ? sh.max_mid : 0, cs);
+    e = launch_select(p, sh.score_tiles > 0 ? sh.max_mid : 0, n_sm_cached(), cs);
   }
   if (e != cudaSuccess) return cuda_fail(e, "select launch");
   {

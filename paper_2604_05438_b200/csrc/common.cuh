@@ -167,7 +167,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // ---------------------------------------------------------------- host launchers
 // Each returns cudaGetLastError() after enqueuing on `stream`.
 cudaError_t launch_score(const Problem& p, const CUtensorMap& tmap_k, int n_sm, cudaStream_t stream);
-cudaError_t launch_select(const Problem& p, int max_mid, cudaStream_t stream);
+cudaError_t launch_select(const Problem& p, int max_mid, int n_sm, cudaStream_t stream);
 cudaError_t launch_exact_residual(const Problem& p, cudaStream_t stream);
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, cudaStream_t stream);
 

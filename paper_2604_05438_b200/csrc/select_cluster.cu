@@ -334,11 +334,17 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
   }
 }
 
-cudaError_t launch_select(const Problem& p, int max_mid, cudaStream_t st) {
+cudaError_t launch_select(const Problem& p, int max_mid, int n_sm, cudaStream_t st) {
   const int rows = p.batch * p.n_q_heads;
-  // cluster size: enough CTAs to keep the longest row in shared memory, at most 8
+  // cluster size: enough CTAs to keep the longest row in shared memory, at most 8 ...
   int csize = 1;
   while (csize < kSelCluster && (long long)csize * kSelChunk < max_mid) csize *= 2;
+  // ... but with many rows the grid fills the GPU several times over anyway, and smaller
+  // clusters (down to one CTA per row, which then reads its row twice) save the cluster
+  // barriers; a CTA handles at most 16 rounds
+  const int n_chunks = (max_mid + kSelChunk - 1) / kSelChunk;
+  while (csize > 1 && (long long)rows * csize > 4LL * n_sm && (n_chunks + csize / 2 - 1) / (csize / 2) <= 16)
+    csize /= 2;
   const int n_tasks = p.with_phi ? rows + p.n_kv_heads : 0;
   const int feat_clusters = (n_tasks + csize - 1) / csize;
   static bool configured = false;
