@@ -19,10 +19,11 @@
 // The k and v rows of a slice are gathered into 128B-swizzled shared-memory tiles.
 // The feature recompute of the retrieved keys, W_k k_i for 128 tokens x r features, is
 // a dense [128 x d] x [d x r] contraction: it runs as tcgen05.mma with the gathered key
-// tile as A and W_k, split into bf16 hi + lo parts (two accumulating MMAs, error
-// ~2^-18 |W|), as B; the 128 x r fp32 result stays in tensor memory and each thread
-// reads the row of its own token, so <phi_q, phi_k(k_i)> needs no cross-thread
-// reduction.  Each CTA writes partial sums; the last CTA of a head (one atomic
+// tile as A and W_k, split into bf16 hi + lo parts (error ~2^-18 |W|) that are stacked
+// into one B operand of 2r rows (an MMA with M = 128 takes the same time for N = 2r as
+// for N = r), as B; the 128 x 2r fp32 result stays in tensor memory and each thread reads
+// the row of its own token and adds the hi and lo halves, so <phi_q, phi_k(k_i)> needs no
+// cross-thread reduction.  Each CTA writes partial sums; the last CTA of a head (one atomic
 // ticket, no spinning) combines them in slice order, so results are run-to-run
 // identical.
 #include "common.cuh"
@@ -37,15 +38,14 @@ template <int D, int R>
 struct ExSmem {
   static constexpr int BOXES = D / 64;
   static constexpr int KV_BOX = kSlice * 128;                 // bytes of one 64-dim column block of k or v
-  static constexpr int W_BOX = R * 128;
+  static constexpr int W_BOX = 2 * R * 128;                   // hi rows, then lo rows
   static constexpr size_t kv_tile = (size_t)BOXES * KV_BOX;   // one k or v tile [BOXES][128][128 B]
   static constexpr size_t kt = 0;                             // bf16 k tiles, one per group
-  static constexpr size_t whi = kt + kExGroups * kv_tile;     // bf16 W_k hi  [BOXES][R][128 B]
-  static constexpr size_t wlo = whi + (size_t)BOXES * W_BOX;
+  static constexpr size_t whi = kt + kExGroups * kv_tile;     // bf16 W_k hi|lo  [BOXES][2R][128 B]
   // the v tiles take over the W_k region once the MMAs have read it (the v rows wait in
   // registers until then)
   static constexpr size_t vt = whi;
-  static constexpr size_t w_bytes = 2 * (size_t)BOXES * W_BOX, v_bytes = kExGroups * kv_tile;
+  static constexpr size_t w_bytes = (size_t)BOXES * W_BOX, v_bytes = kExGroups * kv_tile;
   static constexpr size_t small = whi + (w_bytes > v_bytes ? w_bytes : v_bytes);
   // small: bars[4] (32 B), tok[T] int, isret[T] int, wgt[T], zt[T] (T threads), qf[D], cj[R], spare[R],
   //        red[groups][4*D], misc[32]
@@ -61,7 +61,6 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   unsigned char* kt = smem + L::kt + grp * L::kv_tile;      // this group's tiles
   unsigned char* vt = smem + L::vt + grp * L::kv_tile;
   unsigned char* whi = smem + L::whi;
-  unsigned char* wlo = smem + L::wlo;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::small);   // [0]: W tiles landed, [1 + g]: MMAs of group g done
   int* tok = reinterpret_cast<int*>(bars + 4) + grp * kSlice;        // per-token arrays: this group's part
   int* isret = reinterpret_cast<int*>(bars + 4) + kExThreads + grp * kSlice;
@@ -110,7 +109,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
     *s_abort = 0;
   }
   pdl_wait();                                  // the index lists, features and score rows of the predecessors
-  if (any_ret && warp == 0) tmem_alloc(s_tmem, kExGroups * R);   // after the wait: never hold columns a predecessor needs
+  if (any_ret && warp == 0) tmem_alloc(s_tmem, kExGroups * 2 * R);   // after the wait: never hold columns a predecessor needs
   // ---- 1. token list of this slice
   {
     const int pi = slice * kSlice + gt;
@@ -134,8 +133,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   if (any_ret && tid == 0) {
     const unsigned char* img = reinterpret_cast<const unsigned char*>(p.wk_img + (size_t)kvh * 2 * R * D);
     mbar_expect_tx(&bars[0], 2u * R * D * 2u);
-    bulk_load(whi, img, R * D * 2, &bars[0]);
-    bulk_load(wlo, img + (size_t)R * D * 2, R * D * 2, &bars[0]);
+    bulk_load(whi, img, 2 * R * D * 2, &bars[0]);
   }
 
   // ---- 2. gather rows into swizzled tiles: v always; k for anchors (scores) and, with phi,
@@ -169,20 +167,17 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
     ok = mbar_wait(&bars[0], 0, s_abort);
     if (ok) {
       tc_fence_after_sync();
-      constexpr uint32_t idesc = umma_idesc_bf16(128, R, 0, 0);
+      constexpr uint32_t idesc = umma_idesc_bf16(128, 2 * R, 0, 0);
+      const uint64_t bdesc0 = umma_smem_desc(smem_u32(whi), 16, 1024);
 #pragma unroll
       for (int g = 0; g < kExGroups; ++g) {
         if (!slice_has_ret(slice0 + g)) continue;
-        const uint32_t tmem_d = *s_tmem + g * R;             // group g accumulates in columns [g R, (g+1) R)
+        const uint32_t tmem_d = *s_tmem + g * 2 * R;         // group g: hi part in columns [2gR, 2gR+R), lo part after it
         const uint64_t adesc0 = umma_smem_desc(smem_u32(smem + L::kt + g * L::kv_tile), 16, 1024);
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint64_t bdesc0 = umma_smem_desc(smem_u32(half == 0 ? whi : wlo), 16, 1024);
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k)
-            umma_ss(tmem_d, adesc0 + (uint64_t)(((k >> 2) * L::KV_BOX + (k & 3) * 32) >> 4),
-                    bdesc0 + (uint64_t)(((k >> 2) * L::W_BOX + (k & 3) * 32) >> 4), idesc, (half | k) ? 1u : 0u);
-        }
+        for (int k = 0; k < D / 16; ++k)
+          umma_ss(tmem_d, adesc0 + (uint64_t)(((k >> 2) * L::KV_BOX + (k & 3) * 32) >> 4),
+                  bdesc0 + (uint64_t)(((k >> 2) * L::W_BOX + (k & 3) * 32) >> 4), idesc, k ? 1u : 0u);
         tc_commit(&bars[1 + g]);
       }
     }
@@ -230,16 +225,17 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   }
   if (has_ret && ok) {
     tc_fence_after_sync();
-    const uint32_t tmem_d = *s_tmem + grp * R;
-    // z = 2^(-gamma log2e |k|^2) * sum_j 2^(acc_j + c_j): four partial sums in a fixed order
+    const uint32_t tmem_d = *s_tmem + grp * 2 * R;
+    // z = 2^(-gamma log2e |k|^2) * sum_j 2^(hi_j + lo_j + c_j): four partial sums in a fixed order
     float zp[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int c4 = 0; c4 < R / 32; ++c4) {
-      float v[32];
+      float v[32], vl[32];
       tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, c4 * 32), v);
+      tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, R + c4 * 32), vl);
       tc_wait_ld();
 #pragma unroll
-      for (int j = 0; j < 32; ++j) zp[j & 3] += ex2_approx(v[j] + cj[c4 * 32 + j]);
+      for (int j = 0; j < 32; ++j) zp[j & 3] += ex2_approx((v[j] + vl[j]) + cj[c4 * 32 + j]);
     }
     z_t = ((zp[0] + zp[1]) + (zp[2] + zp[3])) * ex2_approx(-p.gamma_k * kLog2e * kn);
     if (!isret[gt]) z_t = 0.f;
@@ -293,7 +289,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   __syncthreads();
   if (any_ret && warp == 0) {
     tc_fence_after_sync();
-    tmem_dealloc(*s_tmem, kExGroups * R);
+    tmem_dealloc(*s_tmem, kExGroups * 2 * R);
   }
   if (*s_abort) {
     if (tid == 0) atomicExch(p.status, kStatusTimeout);

@@ -104,15 +104,15 @@ __device__ void phi_q_stage2(const Problem& p, int row) {
 }
 
 // W_k of one KV head (fp32 [r][d]), scaled by log2 e so that the recomputed exponents feed
-// exp2 directly -> two bf16 images, hi = bf16(W) and lo = bf16(W - hi),
-// each laid out as the K-major, 128B-swizzled B operand of the feature recompute MMA:
-// [d/64 column blocks][r rows][128 bytes].  By all NT threads of a CTA.
+// exp2 directly -> hi = bf16(W) and lo = bf16(W - hi), stacked into ONE K-major,
+// 128B-swizzled B operand of 2r rows for the feature recompute MMA (rows 0..r-1 hi,
+// rows r..2r-1 lo): [d/64 column blocks][2r rows][128 bytes].  By all NT threads of a CTA.
 template <int NT>
 __device__ void wk_split_job(const Problem& p, int kvh) {
   const int D = p.head_dim, r = p.n_feat;
   const float* W = p.w_k + (size_t)kvh * r * D;
   unsigned char* hi = reinterpret_cast<unsigned char*>(p.wk_img + (size_t)kvh * 2 * r * D);
-  unsigned char* lo = hi + (size_t)r * D * 2;
+  unsigned char* lo = hi + (size_t)r * 128;          // r is a multiple of 8: the swizzle phase of a row is kept
   const int cpr = D / 8;
 #pragma unroll 4
   for (int i = threadIdx.x; i < r * cpr; i += NT) {
@@ -130,7 +130,7 @@ __device__ void wk_split_job(const Problem& p, int kvh) {
       hw[e] = (unsigned)__bfloat16_as_ushort(h0) | ((unsigned)__bfloat16_as_ushort(h1) << 16);
       lw[e] = (unsigned)__bfloat16_as_ushort(l0) | ((unsigned)__bfloat16_as_ushort(l1) << 16);
     }
-    const size_t off = (size_t)(c >> 3) * r * 128 + swz128(row, c & 7);
+    const size_t off = (size_t)(c >> 3) * (2 * r) * 128 + swz128(row, c & 7);
     *reinterpret_cast<uint4*>(hi + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
     *reinterpret_cast<uint4*>(lo + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
   }
