@@ -179,6 +179,33 @@ tkphi_status make_tensor_map(const tkphi_kv_desc* kv, const void* base, int box_
   return TKPHI_OK;
 }
 
+// 2-D view [row][dim] of a K or V cache for TMA row gathers: box = one row of 64 dims, 128-byte
+// swizzle.  Possible when the rows of all heads lie on one pitch: head-major caches
+// (stride_head a multiple of stride_token: row = head * ratio + token) or token-major ones
+// (stride_token a multiple of stride_head: row = token * ratio + head).  Returns the mode
+// (-1: not expressible; the kernel then gathers with 16-byte copies).
+int make_gather_map(const tkphi_kv_desc* kv, const void* base, long long total_tokens, CUtensorMap* tm,
+                    long long* ratio, long long* rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return -1;
+  const long long sh = kv->kv_stride_head, stt = kv->kv_stride_token, H = kv->n_kv_heads;
+  int mode;
+  long long pitch;
+  if (H == 1) { mode = 0; *ratio = total_tokens; pitch = stt; *rows = total_tokens; }
+  else if (sh % stt == 0 && sh / stt >= total_tokens) { mode = 0; *ratio = sh / stt; pitch = stt; *rows = (H - 1) * *ratio + total_tokens; }
+  else if (stt % sh == 0 && stt / sh >= H) { mode = 1; *ratio = stt / sh; pitch = sh; *rows = (total_tokens - 1) * *ratio + H; }
+  else return -1;
+  if (pitch < kv->head_dim || (pitch * 2) % 16 != 0 || *rows >= (1LL << 31) - 1 || *rows < 1) return -1;
+  const cuuint64_t dims[2] = {(cuuint64_t)kv->head_dim, (cuuint64_t)*rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+  const cuuint32_t box[2] = {64, 1};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? mode : -1;
+}
+
 // ---- optional per-kernel timing (off by default): CUDA events around every launch
 struct TimedSpan { cudaEvent_t a, b; int kind; };
 bool g_timing = false;
@@ -290,7 +317,26 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   if (e != cudaSuccess) return cuda_fail(e, "select launch");
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_EXACT_RESIDUAL);
-    e = launch_exact_residual(p, cs);
+    // slice pairs of the whole call (two 128-token slices of a support list per CTA)
+    long long n_pairs = 0;
+    for (int b = 0; b < kv->batch; ++b) {
+      const long long len_b = kv->cu_seqlens_host[b + 1] - kv->cu_seqlens_host[b];
+      const long long n_a1 = len_b < kv->n_sink ? len_b : kv->n_sink;
+      long long ts = len_b - kv->n_tail;
+      if (ts < kv->n_sink) ts = kv->n_sink;
+      if (ts > len_b) ts = len_b;
+      const long long n_e = n_a1 + topk_host[b] + (len_b - ts);
+      const long long n_slices = n_e > 0 ? (n_e + kSlice - 1) / kSlice : 1;
+      n_pairs += (long long)kv->n_q_heads * ((n_slices + 1) / 2);
+    }
+    CUtensorMap gk, gv;
+    memset(&gk, 0, sizeof(gk));
+    memset(&gv, 0, sizeof(gv));
+    long long ratio_v = 0, rows_v = 0;
+    p.gather_mode = make_gather_map(kv, kv->k, sh.total_tokens, &gk, &p.gather_ratio, &p.gather_rows);
+    if (p.gather_mode >= 0 && make_gather_map(kv, kv->v, sh.total_tokens, &gv, &ratio_v, &rows_v) != p.gather_mode)
+      p.gather_mode = -1;
+    e = launch_exact_residual(p, gk, gv, n_pairs, n_sm_cached(), cs);
   }
   if (e != cudaSuccess) return cuda_fail(e, "exact_residual launch");
   return TKPHI_OK;

@@ -36,6 +36,10 @@ struct Problem {
   float gamma_q, gamma_k;
   // summaries
   const float* S; const float* u;
+  // row gather of the exact support through 2-D tensor maps over the k and v caches:
+  // gather_mode 0: row = kv head * gather_ratio + cache row; 1: row = cache row * gather_ratio + kv head;
+  // -1: the cache strides do not form a 2-D tensor, rows are gathered with 16-byte copies
+  int gather_mode; long long gather_ratio; long long gather_rows;
   // outputs
   int* idx_out; float* y_out; float* dbg_out;
   unsigned flags;
@@ -168,7 +172,8 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // Each returns cudaGetLastError() after enqueuing on `stream`.
 cudaError_t launch_score(const Problem& p, const CUtensorMap& tmap_k, int n_sm, cudaStream_t stream);
 cudaError_t launch_select(const Problem& p, int max_mid, int n_sm, cudaStream_t stream);
-cudaError_t launch_exact_residual(const Problem& p, cudaStream_t stream);
+cudaError_t launch_exact_residual(const Problem& p, const CUtensorMap& gk, const CUtensorMap& gv, long long n_pairs, int n_sm,
+                                  cudaStream_t stream);
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, cudaStream_t stream);
 
 }  // namespace tkphi

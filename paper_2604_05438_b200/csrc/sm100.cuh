@@ -96,6 +96,17 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, ui
       "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(l2_policy)
       : "memory");
 }
+// Row gather: four rows (r0..r3, any order, out-of-range rows read as zeros) of a 2-D
+// tensor, `col` .. `col` + box width of each, land as four consecutive 128-byte rows at dst
+// (the tensor map's box is one row high and 128 bytes wide, 128B swizzle).
+__device__ __forceinline__ void tma_gather4_2d(void* dst, const CUtensorMap* tm, uint64_t* bar, int col, int r0,
+                                               int r1, int r2, int r3, uint64_t l2_policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;" ::"r"(smem_u32(dst)),
+      "l"(tm), "r"(smem_u32(bar)), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "l"(l2_policy)
+      : "memory");
+}
 // Untiled bulk copy global -> shared; both addresses 16-byte aligned, bytes % 16 == 0.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile(

@@ -156,6 +156,23 @@ def test_c4_ragged_batch():
     _check_decode(gl, 0, 0.05, None, None, with_phi=False, topk=topk)
 
 
+def test_many_rows_take_the_streaming_exact_kernel():
+    # 8 sequences x 24 query heads = 192 rows, each at least one slice pair: more pairs than SMs at
+    # head_dim 128, so the persistent, software-pipelined exact/residual kernel runs (items of
+    # different length, KV head changes and sequence boundaries inside a CTA's range)
+    cfg = _cfg("c3_3b_128k", batch=8, needle_every=256)
+    inp = make_layer_inputs(cfg, 7, seq_lens=[900, 300, 133, 1500, 700, 2049, 132, 1100], n_steps=1)
+    phi0 = make_phi_params(cfg, 7, kind="visible")
+    phi = make_phi_params(cfg, 7, kind="visible", bk_shift=PU.calibrate_visible_shift(cfg, inp, phi0, 0.2))
+    gl = PU.to_gpu(cfg, inp, phi)
+    S, u = PU.gpu_build(gl)
+    topk = inp.topk(0.2)
+    assert int(topk.max()) > 256 and int(topk.min()) == 0      # several slice pairs for some heads, none retrieved for others
+    _check_decode(gl, 0, 0.2, S, u, topk=topk, heads=range(0, 24, 5))
+    _check_decode(gl, 0, 0.2, S, u, topk=topk, flags=1, heads=[1, 22])
+    _check_decode(gl, 0, 0.2, None, None, with_phi=False, topk=topk, heads=[2, 17])
+
+
 def test_c5_zipf_norms_reduced_length():
     cfg = _cfg("c5_3b_1m", batch=2)
     inp = make_layer_inputs(cfg, 1, seq_lens=[6000, 3001], n_steps=1)
