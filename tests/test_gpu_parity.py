@@ -156,11 +156,12 @@ def test_c4_ragged_batch():
     _check_decode(gl, 0, 0.05, None, None, with_phi=False, topk=topk)
 
 
-def test_many_rows_take_the_streaming_exact_kernel():
+@pytest.mark.parametrize("n_feat", [128, 64])
+def test_many_rows_take_the_streaming_exact_kernel(n_feat):
     # 8 sequences x 24 query heads = 192 rows, each at least one slice pair: more pairs than SMs at
     # head_dim 128, so the persistent, software-pipelined exact/residual kernel runs (items of
     # different length, KV head changes and sequence boundaries inside a CTA's range)
-    cfg = _cfg("c3_3b_128k", batch=8, needle_every=256)
+    cfg = _cfg("c3_3b_128k", batch=8, needle_every=256, n_feat=n_feat)
     inp = make_layer_inputs(cfg, 7, seq_lens=[900, 300, 133, 1500, 700, 2049, 132, 1100], n_steps=1)
     phi0 = make_phi_params(cfg, 7, kind="visible")
     phi = make_phi_params(cfg, 7, kind="visible", bk_shift=PU.calibrate_visible_shift(cfg, inp, phi0, 0.2))
@@ -171,6 +172,30 @@ def test_many_rows_take_the_streaming_exact_kernel():
     _check_decode(gl, 0, 0.2, S, u, topk=topk, heads=range(0, 24, 5))
     _check_decode(gl, 0, 0.2, S, u, topk=topk, flags=1, heads=[1, 22])
     _check_decode(gl, 0, 0.2, None, None, with_phi=False, topk=topk, heads=[2, 17])
+
+
+@pytest.mark.parametrize("layout", ["token_major", "padded_heads"])
+def test_streaming_exact_kernel_other_cache_layouts(layout):
+    # token-major caches gather rows as token * H + head; a cache whose head stride is not a multiple of
+    # its token stride has no 2-D row view: the call then runs the one-shot kernel with 16-byte copies
+    import paper_2604_05438_b200 as T
+    cfg = _cfg("c3_3b_128k", batch=8, needle_every=256)
+    inp = make_layer_inputs(cfg, 8, seq_lens=[900, 300, 133, 1500, 700, 2049, 132, 1100], n_steps=1)
+    phi = make_phi_params(cfg, 8)
+    gl = PU.to_gpu(cfg, inp, phi, token_major=(layout == "token_major"))
+    if layout == "padded_heads":
+        H, Tn, d = inp.k.shape
+        def padded(x):
+            store = torch.zeros(H, Tn * d + 8, dtype=x.dtype, device=gl.dev)
+            view = store[:, : Tn * d].view(H, Tn, d)
+            view.copy_(x.to(gl.dev))
+            return view
+        k, v = padded(inp.k), padded(inp.v)
+        assert k.stride(0) == Tn * d + 8
+        gl.kv = T.KVCache(k, v, inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, inp.n_sink, inp.n_tail)
+    S, u = PU.gpu_build(gl)
+    topk = inp.topk(0.2)
+    _check_decode(gl, 0, 0.2, S, u, topk=topk, heads=[0, 7, 23])
 
 
 def test_c5_zipf_norms_reduced_length():
