@@ -198,6 +198,17 @@ def test_streaming_exact_kernel_other_cache_layouts(layout):
     _check_decode(gl, 0, 0.2, S, u, topk=topk, heads=[0, 7, 23])
 
 
+def test_one_cta_row_budgets_from_one_key_to_half_the_row():
+    # a row of 8192..16384 mid keys is selected by a single CTA; budgets from one key to half of the
+    # row, needles give exact ties at the threshold
+    cfg = _cfg("c1_1b_4k", needle_every=300)
+    inp = make_layer_inputs(cfg, 9, seq_lens=[12000], n_steps=1)
+    gl = PU.to_gpu(cfg, inp, make_phi_params(cfg, 9))
+    n_mid = 12000 - inp.n_sink - inp.n_tail
+    for k in (1, 119, n_mid // 8, n_mid // 8 + 1, n_mid // 2):
+        _check_decode(gl, 0, 0.0, None, None, with_phi=False, topk=[k], heads=[0, 5, 31])
+
+
 def test_c5_zipf_norms_reduced_length():
     cfg = _cfg("c5_3b_1m", batch=2)
     inp = make_layer_inputs(cfg, 1, seq_lens=[6000, 3001], n_steps=1)
