@@ -638,16 +638,42 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
   if (do_phi && warp == 0) tmem_alloc(s_tmem, kExGroups * 2 * R);
   ExItem cur = item_of(i0, nullptr);
   if (!producer) stage_store(stage_load(cur), 0);
+  if (tid == 0) {                              // the first item's tiles: announced here, issued by all compute warps below
+    mbar_expect_tx(&bars[3], (uint32_t)(kExGroups * LB::kv_tile));
+    mbar_expect_tx(&bars[4], (uint32_t)(kExGroups * LB::kv_tile));
+  }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
+  // The gathers of the first item are on every CTA's critical path, and one warp needs about
+  // 4.5 us to issue the 128 gathers of a tile pair: here each of the eight compute warps
+  // issues one (k or v, group, column block) combination, one gather per lane.
+  if (!producer) {
+    static_assert(kExGroups * LB::BOXES * 2 == kExThreads / 32, "one (kind, group, column block) per compute warp");
+    const bool keys = warp < kExThreads / 64;
+    const int g = (warp / LB::BOXES) % kExGroups, x = warp % LB::BOXES;
+    const int* tk = tok_all + g * kSlice;
+    const int* ir = isret_all + g * kSlice;
+    int r[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int t = 4 * lane + j;
+      const int ti = tk[t];
+      const bool want = ti >= 0 && (!keys || !ir[t] || do_phi);
+      const long long cache_row = cur.cu_b + ti;
+      const long long gr = p.gather_mode == 0 ? (long long)cur.kvh * p.gather_ratio + cache_row
+                                              : cache_row * p.gather_ratio + cur.kvh;
+      r[j] = want ? (int)gr : (int)p.gather_rows;
+    }
+    tma_gather4_2d(smem + (keys ? L::kt : L::vt) + g * LB::kv_tile + x * LB::KV_BOX + 4 * lane * 128,
+                   keys ? &gmap_k : &gmap_v, &bars[keys ? 3 : 4], x * 64, r[0], r[1], r[2], r[3], pol);
+  }
 
   if (producer) {
     // ================================================================ row-gather producers
     const bool keys = warp == kExThreads / 32;
     uint64_t* free_bar = &bars[keys ? 5 : 6];
-    issue_rows(cur, 0, keys);
-    int issued = 1;
+    int issued = 1;                            // (the first item's gathers were issued by the compute warps)
     for (int i = i0; i + 1 < i1; ++i) {
       const ExItem nx = item_of(i + 1, &cur);
       // the compute warps are done with the tiles of item i (and have staged item i+1's token list)
