@@ -49,7 +49,7 @@ extern "C" {
 typedef enum {
   TKPHI_OK = 0,
   TKPHI_ERR_INVALID_ARG = -1,  /* bad pointer, size, stride or range */
-  TKPHI_ERR_UNSUPPORTED = -2,  /* legal problem this build has no kernel for */
+  TKPHI_ERR_UNSUPPORTED = -2,  /* legal problem the library has no kernel for */
   TKPHI_ERR_WORKSPACE = -3,    /* workspace NULL, misaligned or too small */
   TKPHI_ERR_CUDA = -4,         /* a CUDA runtime/driver call failed */
   TKPHI_ERR_TIMEOUT = -5       /* a bounded device-side wait ran out (see tkphi_device_status) */
@@ -75,6 +75,10 @@ enum {
  * both strides multiples of 8 elements; kv_stride_token >= head_dim; total rows
  * < 2^31; at most 2,097,152 mid-region rows per sequence for the decode entry points.
  * Query head h_q uses KV head h_q / (n_q_heads / n_kv_heads).
+ * Any strides within these rules work.  Head-major caches (kv_stride_head a multiple of
+ * kv_stride_token) and token-major ones (kv_stride_token a multiple of kv_stride_head) also
+ * let the decode entry points fetch the rows of the exact support by TMA row gathers, which
+ * calls with many retrieved rows (more 256-token pieces of support lists than SMs) use.
  * Anchors (Eq. partition): the first n_sink and the last n_tail rows of each
  * sequence (their union when L_b < n_sink + n_tail); the mid-region is what lies
  * between, |M_b| = max(0, L_b - n_sink - n_tail).
