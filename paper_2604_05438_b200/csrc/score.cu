@@ -6,8 +6,10 @@
 //                  128B-swizzled 32 KB key tiles into a 3-stage mbarrier ring; one thread
 //                  issues tcgen05.mma with the key tile as an operand straight from shared
 //                  memory and the group's queries (zero padded) as the other, so the dot
-//                  products cost no issue slots of the CUDA cores; one warp reads the fp32
-//                  accumulators back from tensor memory and writes the score rows.  The
+//                  products cost no issue slots of the CUDA cores; two warps (even and odd
+//                  tiles) read the fp32 accumulators back from tensor memory and write the
+//                  score rows (with one warp that stage bounds the kernel at head_dim 64,
+//                  where a tile holds 256 keys of four heads).  The
 //                  CTAs also clear the workspace counters.
 #include "common.cuh"
 #include "sm100.cuh"
@@ -15,7 +17,9 @@
 namespace tkphi {
 
 // ------------------------------------------------------------------ scoring
-constexpr int kScoreThreads = 96;         // warp 0: read-back, warp 1: MMA issuer, warp 2: TMA producer
+constexpr int kScoreThreads = 160;        // warps 0 and 4: read-back (even / odd tiles; a warp reads tensor-memory lanes
+                                          // 32 (w % 4) .. + 31 and the scores sit in lanes 0..15), warp 1: MMA issuer,
+                                          // warp 2: TMA producer, warp 3 idle
 constexpr int kScoreStages = 3;          // measured: 3-4 stages beat 6 (less queueing in the memory system)
 constexpr int kScoreTileBytes = 32768;
 constexpr int kScoreM = 64;               // MMA M: query heads of the group (<= 8), zero padded
@@ -232,7 +236,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         cursor_next(mc, pre, batch, n_kv);
       }
-    } else {
+    } else if (warp == 0 || warp == 4) {
       // ================================================================ read-back, score rows
       // warp 0 reads tensor-memory lanes 0..15: thread t holds head (t / 4), key columns
       // 8 i + 2 (t % 4) + {0, 1} of each 8-column block i (the second register pair of a
@@ -253,6 +257,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
           n_mid = mid_len(len_b, p.n_sink, p.n_tail);
           my_row = p.scores + score_row_base(p, cur_b, cur_kvh * G, cu_b, len_b) + (long long)g * len_b;
         }
+        if ((it & 1) != (warp >> 2)) { cursor_next(cc, pre, batch, n_kv); continue; }   // the other read-back warp's tile
         const int a = it % ACC;
         const uint32_t aph = (uint32_t)(it / ACC) & 1u;
         ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[a], aph, s_abort));
