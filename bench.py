@@ -46,7 +46,7 @@ def _peaks():
 
 # DRAM bytes per launch of the scoring kernel from the committed ncu capture of this kernel
 # (profiles/); None once the kernel has changed since the capture.
-SCORE_KERNEL_NCU_TRAFFIC_BYTES = 268231168 + 3602176    # dram read + write, profiles/decode_kernels_c3_one_layer.md
+SCORE_KERNEL_NCU_TRAFFIC_BYTES = 268231936 + 3233792    # dram read + write, profiles/decode_kernels_c3_one_layer.md
 
 
 # --------------------------------------------------------------------------- clocks
