@@ -33,6 +33,7 @@ struct ScoreCfg {
   static constexpr int QBOX_BYTES = kScoreM * 128;
   static constexpr int ACC_STAGES = kTmemCols / TK;      // accumulator buffers in tensor memory
   static_assert(TK * D * 2 == kScoreTileBytes && TK <= 256, "tile size");
+  static_assert(ACC_STAGES % 2 == 0, "two read-back warps alternate over the accumulator buffers");
 };
 
 struct TileCursor {
@@ -257,7 +258,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
           n_mid = mid_len(len_b, p.n_sink, p.n_tail);
           my_row = p.scores + score_row_base(p, cur_b, cur_kvh * G, cu_b, len_b) + (long long)g * len_b;
         }
-        if ((it & 1) != (warp >> 2)) { cursor_next(cc, pre, batch, n_kv); continue; }   // the other read-back warp's tile
+        // the other read-back warp's tile (every accumulator buffer belongs to one warp: their number is even)
+        if ((it & 1) != (warp >> 2)) { cursor_next(cc, pre, batch, n_kv); continue; }
         const int a = it % ACC;
         const uint32_t aph = (uint32_t)(it / ACC) & 1u;
         ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[a], aph, s_abort));
