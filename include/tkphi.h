@@ -74,6 +74,10 @@ enum {
  * n_kv_heads with group size <= 8; n_feat in {64, 128}; k and v 16-byte aligned;
  * both strides multiples of 8 elements; kv_stride_token >= head_dim; total rows
  * < 2^31; at most 2,097,152 mid-region rows per sequence for the decode entry points.
+ * With more than one KV head the heads must not share memory: either kv_stride_head >=
+ * rows * kv_stride_token (head-major) or kv_stride_head >= head_dim and kv_stride_token >=
+ * (n_kv_heads - 1) * kv_stride_head + head_dim (token-major); anything else, a zero head
+ * stride included, is TKPHI_ERR_INVALID_ARG.
  * Query head h_q uses KV head h_q / (n_q_heads / n_kv_heads).
  * Any strides within these rules work.  Head-major caches (kv_stride_head a multiple of
  * kv_stride_token) and token-major ones (kv_stride_token a multiple of kv_stride_head) also
@@ -137,21 +141,32 @@ tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc
  *  - Limit: problems whose tkphi_workspace_bytes(kv, NULL, 0, TKPHI_WS_BUILD) exceeds
  *    TKPHI_STATIC_SCRATCH_BYTES are rejected with TKPHI_ERR_WORKSPACE before anything
  *    is enqueued (the message names both sizes); use tkphi_build_summaries for those.
- *  - Cost: every GPU on which the library is loaded holds the array until the process
- *    exits, whether or not this function is ever called.
+ *  - Cost: the array is part of the library's device code.  Every GPU on which that code
+ *    is loaded holds the array until the process exits.  The CUDA runtime loads it on a
+ *    device when the library is first used there (at the latest by this function's first
+ *    call on the device, which therefore is also where the device's free memory drops by
+ *    the array's size).
  *  - First call on each device: looks up the array's device address (a host-side
  *    runtime query, done with that device current and cached).  Make that first call
- *    before any stream capture begins on the device.
+ *    at initialisation, before any stream capture begins on the device.
  *  - Sharing: all calls on a device use the same array.  The array keeps the previous
- *    call's contents; the part that must start at zero is cleared on the stream at the
- *    start of every call.  Two calls whose GPU work overlaps (different streams, or
- *    different host threads) race on it and give undefined results: serialise them.
+ *    call's contents; the build needs none of it cleared (the kernel sets the status word
+ *    at the head of the array itself and overwrites every partial sum before it is read).
+ *    Two calls whose GPU work overlaps (different streams, or different host threads)
+ *    race on it and give undefined results: serialise them.
+ *  - Device-side errors: tkphi_static_device_status reads the status word of the last
+ *    static call on the current device (the array's address is not exposed, so
+ *    tkphi_device_status cannot be used): 0, or TKPHI_ERR_TIMEOUT if a bounded wait of the
+ *    build kernel ran out, in which case (S, u) are not valid.  Waits for the stream;
+ *    *status_out is a host int.  TKPHI_ERR_INVALID_ARG if no static call has been made on
+ *    the device yet.
  * Arguments, outputs and error reporting otherwise as for tkphi_build_summaries;
  * tkphi_static_last_error() gives the message of the last failing call of the thread.
  */
 #define TKPHI_STATIC_SCRATCH_BYTES (8u << 20)
 tkphi_status tkphi_build_summaries_static(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi,
                                           float* S, float* u, void* cuda_stream);
+tkphi_status tkphi_static_device_status(void* cuda_stream, int32_t* status_out);
 const char* tkphi_static_last_error(void);
 
 /*
@@ -206,6 +221,21 @@ tkphi_status tkphi_decode_step(const tkphi_kv_desc* kv, const tkphi_phi_desc* ph
 tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32_t* status_out);
 
 /*
+ * Self-test of the error path of the bounded device-side waits (no counterpart in the
+ * paper).  Every wait inside the kernels (on a TMA copy, an MMA completion, a hand-off
+ * between warps) gives up after a fixed number of polls, raises a flag that makes the
+ * other warps of its CTA leave their loops, and the CTA stores TKPHI_ERR_TIMEOUT in the
+ * status word at the head of the workspace before it returns.  This entry point runs a
+ * one-CTA kernel through exactly that path: one warp waits, with a limit of 4096 polls, on
+ * a barrier that nothing ever arrives on, a second warp waits on a barrier the first one
+ * would have signalled.  The kernel returns by itself within microseconds; afterwards
+ * tkphi_device_status(workspace) reads TKPHI_ERR_TIMEOUT, and the next ordinary call on
+ * the same workspace sets the word back to 0.  workspace: device memory, 256-byte
+ * aligned, at least 256 bytes.
+ */
+tkphi_status tkphi_selftest_timeout(void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Optional per-kernel timing for benchmarks (no counterpart in the paper).  While
  * enabled, every launch the library makes is bracketed by CUDA events on the caller's
  * stream (the events are host objects; no device memory is allocated).  Not
@@ -215,13 +245,11 @@ tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32
  */
 enum {
   TKPHI_KERNEL_SCORE = 0,           /* key scoring (streams the mid-region keys) */
-  TKPHI_KERNEL_RESERVED_1 = 1,
-  TKPHI_KERNEL_SELECT = 2,          /* exact Top-K over the score rows; query-side feature work */
-  TKPHI_KERNEL_EXACT_RESIDUAL = 3,  /* exact branch, subtraction, residual, merge */
-  TKPHI_KERNEL_BUILD = 4,           /* prefill summary build */
-  TKPHI_KERNEL_MEMSET = 5,          /* clearing counters when there is nothing to score */
-  TKPHI_KERNEL_RESERVED_6 = 6,
-  TKPHI_KERNEL_KINDS = 7
+  TKPHI_KERNEL_SELECT = 1,          /* exact Top-K over the score rows; query-side feature work */
+  TKPHI_KERNEL_EXACT_RESIDUAL = 2,  /* exact branch, subtraction, residual, merge */
+  TKPHI_KERNEL_BUILD = 3,           /* prefill summary build */
+  TKPHI_KERNEL_MEMSET = 4,          /* clearing counters when there is nothing to score */
+  TKPHI_KERNEL_KINDS = 5
 };
 void tkphi_kernel_timing_enable(int32_t on);
 tkphi_status tkphi_kernel_timing_read(float* ms_out, int32_t* count_out);

@@ -18,6 +18,9 @@ from .binding import (  # noqa: F401
     topk_decode,
     decode_step,
     device_status,
+    static_device_status,
+    selftest_timeout,
+    ERR_TIMEOUT,
     kernel_timing,
     KERNEL_KINDS,
     WS_BUILD,

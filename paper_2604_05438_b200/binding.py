@@ -20,10 +20,12 @@ EXPORTED_SYMBOLS = (
     "tkphi_workspace_bytes", "tkphi_build_summaries", "tkphi_topk_decode", "tkphi_decode_step",
     "tkphi_device_status", "tkphi_last_error", "tkphi_version",
     "tkphi_kernel_timing_enable", "tkphi_kernel_timing_read",
-    "tkphi_build_summaries_static", "tkphi_static_last_error",
+    "tkphi_build_summaries_static", "tkphi_static_last_error", "tkphi_static_device_status",
+    "tkphi_selftest_timeout",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
-KERNEL_KINDS = ("score", "reserved_1", "select", "exact_residual", "build", "memset", "reserved_6")
+KERNEL_KINDS = ("score", "select", "exact_residual", "build", "memset")
+ERR_TIMEOUT = -5
 
 
 class TkphiError(RuntimeError):
@@ -67,6 +69,10 @@ def load_library():
     lib.tkphi_build_summaries_static.argtypes = [C.POINTER(_KvDesc), C.POINTER(_PhiDesc), C.c_void_p, C.c_void_p,
                                                  C.c_void_p]
     lib.tkphi_static_last_error.restype = C.c_char_p
+    lib.tkphi_static_device_status.restype = C.c_int
+    lib.tkphi_static_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+    lib.tkphi_selftest_timeout.restype = C.c_int
+    lib.tkphi_selftest_timeout.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
     lib.tkphi_topk_decode.restype = C.c_int
     lib.tkphi_topk_decode.argtypes = [C.POINTER(_KvDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -185,6 +191,23 @@ def build_summaries_static(kv: KVCache, phi: PhiMaps, S: torch.Tensor, u: torch.
     st = lib.tkphi_build_summaries_static(C.byref(d), C.byref(ph), S.data_ptr(), u.data_ptr(), _stream_ptr(stream))
     if st != 0:
         raise TkphiError(st, lib.tkphi_static_last_error().decode())
+
+
+def static_device_status(stream=None) -> int:
+    """Status word of the last build_summaries_static call on the current device (0 = fine)."""
+    lib = load_library()
+    out = C.c_int32(0)
+    st = lib.tkphi_static_device_status(_stream_ptr(stream), C.byref(out))
+    if st != 0:
+        raise TkphiError(st, lib.tkphi_static_last_error().decode())
+    return int(out.value)
+
+
+def selftest_timeout(workspace: torch.Tensor, stream=None) -> None:
+    """Runs the library's bounded-wait self-test kernel; device_status(workspace) then reads ERR_TIMEOUT."""
+    lib = load_library()
+    _check(lib.tkphi_selftest_timeout(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                      _stream_ptr(stream)))
 
 
 def topk_decode(kv: KVCache, q: torch.Tensor, topk_host, topk_dev: torch.Tensor, topk_max: int,

@@ -68,6 +68,18 @@ tkphi_status validate_kv(const tkphi_kv_desc* kv, Shape* sh, bool need_data) {
     if (kv->kv_stride_token < kv->head_dim || kv->kv_stride_token % 8 != 0 || kv->kv_stride_head % 8 != 0 ||
         kv->kv_stride_head < 0)
       return fail(TKPHI_ERR_INVALID_ARG, "strides must be multiples of 8 elements, token stride >= head_dim");
+    if (kv->n_kv_heads > 1) {
+      // rows of different heads must not share memory: head-major (a head's rows come before the
+      // next head's) or token-major (the heads of one token come before the next token's)
+      const long long sth = kv->kv_stride_head, stt = kv->kv_stride_token;
+      const bool head_major = sth >= sh->total_tokens * stt;
+      const bool token_major = sth >= kv->head_dim && stt >= (long long)(kv->n_kv_heads - 1) * sth + kv->head_dim;
+      if (!head_major && !token_major)
+        return fail(TKPHI_ERR_INVALID_ARG,
+                    "kv_stride_head = %lld with %d KV heads: the heads overlap (need kv_stride_head >= rows * "
+                    "kv_stride_token, or kv_stride_head >= head_dim and kv_stride_token >= (n_kv_heads - 1) * "
+                    "kv_stride_head + head_dim)", sth, kv->n_kv_heads);
+    }
   }
   return TKPHI_OK;
 }
@@ -97,15 +109,7 @@ tkphi_status validate_topk(const tkphi_kv_desc* kv, const int32_t* topk_host, in
   return TKPHI_OK;
 }
 
-int n_sm_cached() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
+int n_sm_cached() { return sm_count_current_device(); }
 
 void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, WsLayout* L) {
   size_t o = 0;
@@ -128,14 +132,12 @@ void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, W
 void build_layout(const tkphi_kv_desc* kv, const Shape& sh, WsLayout* L) {
   size_t o = 0;
   L->status = o;        o += 256;
-  L->unit_counter = o;  o = align_up(o + sizeof(unsigned) * sh.units, 256);
   L->zero_end = o;
   // one CTA per SM over all units, never more chunks than 128-token tiles
   const int64_t max_tiles = sh.max_mid > 0 ? ((int64_t)sh.max_mid + 127) / 128 : 1;
   int64_t cpu = n_sm_cached() / sh.units;
   if (cpu < 1) cpu = 1;
   if (cpu > max_tiles) cpu = max_tiles;
-  L->chunk_len = 0;
   L->chunks_per_unit = (int)cpu;
   L->b_partials = o;
   o = align_up(o + sizeof(float) * (size_t)sh.units * L->chunks_per_unit *
@@ -169,9 +171,10 @@ tkphi_status make_tensor_map(const tkphi_kv_desc* kv, const void* base, int box_
   const cuuint64_t strides[2] = {(cuuint64_t)kv->kv_stride_token * 2, (cuuint64_t)kv->kv_stride_head * 2};
   const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};   // 128-byte rows
   const cuuint32_t estr[3] = {1, 1, 1};
-  // a single head (stride 0 would be rejected): give the unused dimension a legal stride
+  // a single head (any stride is legal for the caller, the encoder rejects 0): give the unused
+  // dimension a legal stride
   cuuint64_t st[2] = {strides[0], strides[1]};
-  if (kv->n_kv_heads == 1 || st[1] == 0) st[1] = st[0] * (cuuint64_t)total_tokens;
+  if (kv->n_kv_heads == 1) st[1] = st[0] * (cuuint64_t)total_tokens;
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, st, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -344,6 +347,33 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
 
 }  // namespace
 
+namespace tkphi {
+
+int sm_count_current_device() {
+  static int n_sm[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  if (n_sm[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    n_sm[dev] = n;
+  }
+  return n_sm[dev];
+}
+
+cudaError_t set_max_dynamic_smem(PerDeviceFlag& flag, const void* kernel, size_t bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < kMaxDevices;
+  if (tracked && flag.done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess && tracked) flag.done[dev] = true;
+  return e;
+}
+
+}  // namespace tkphi
+
 extern "C" {
 
 const char* tkphi_last_error(void) { return g_err; }
@@ -391,9 +421,8 @@ tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc
   p.w_k = phi->w_k; p.b_k = phi->b_k; p.gamma_k = phi->gamma_k;
   p.S = S; p.u = u;
   p.status = reinterpret_cast<int*>(w + L.status);
-  p.unit_counter = reinterpret_cast<unsigned*>(w + L.unit_counter);
   p.partials = reinterpret_cast<float*>(w + L.b_partials);
-  p.chunk_len = L.chunk_len; p.chunks_per_unit = L.chunks_per_unit;
+  p.chunks_per_unit = L.chunks_per_unit;
   if (!aligned16(phi->w_k)) return fail(TKPHI_ERR_INVALID_ARG, "w_k must be 16-byte aligned");
   CUtensorMap tk, tv;
   st = make_tensor_map(kv, kv->k, 128, sh.total_tokens, &tk);

@@ -374,16 +374,13 @@ __global__ void __launch_bounds__(kRedThreads) build_reduce_kernel(const BuildPr
 template <int D>
 static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, const CUtensorMap& tv,
                                   cudaStream_t st) {
-  static bool configured = false;
+  static PerDeviceFlag configured;
   const size_t smem = BuildCfg<D>::total;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(build_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e = set_max_dynamic_smem(configured, reinterpret_cast<const void*>(build_kernel<D>), smem);
+  if (e != cudaSuccess) return e;
   dim3 grid(p.chunks_per_unit, p.n_kv_heads, p.batch);
   build_kernel<D><<<grid, kBuildThreads, smem, st>>>(tk, tv, p);
-  cudaError_t e = cudaGetLastError();
+  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   // one output per thread: every thread's loads of all chunk partials are in flight at once
   const int n_out = p.head_dim * p.n_feat + p.n_feat;

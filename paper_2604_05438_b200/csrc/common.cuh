@@ -66,19 +66,17 @@ struct BuildProblem {
   const float* w_k; const float* b_k; float gamma_k;
   float* S; float* u;
   int* status;
-  unsigned* unit_counter;          // [batch*n_kv_heads]
   float* partials;                 // [units][chunks_per_unit][d*r + r]
-  int chunk_len;                   // unused
   int chunks_per_unit;             // upper bound over sequences
 };
 
 // Host-side byte offsets of the workspace pieces.
 struct WsLayout {
-  size_t status, unit_counter, row_counter, zero_end;
+  size_t status, row_counter, zero_end;
   size_t scores, wk_img, idx, aq, partials, total;
   int max_slices, partial_stride;
   // build
-  size_t b_partials; int chunk_len, chunks_per_unit;
+  size_t b_partials; int chunks_per_unit;
 };
 
 // Row length of Problem::aq: [0, r) w; [r] m_q; [r+1] w.u_M; [r+4, r+4+d) S_M w; [r+4+d, 2r+4+d) log2 w.
@@ -167,6 +165,16 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.attrs = attr; cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+
+// ---------------------------------------------------------------- per-device host state
+// A process may drive several GPUs: what is configured or queried per device is kept per
+// device ordinal of the calling thread's current device.
+constexpr int kMaxDevices = 64;
+struct PerDeviceFlag { bool done[kMaxDevices] = {}; };
+// cudaFuncAttributeMaxDynamicSharedMemorySize of `kernel`, set once on the current device.
+cudaError_t set_max_dynamic_smem(PerDeviceFlag& flag, const void* kernel, size_t bytes);
+// Multiprocessor count of the current device (148 if it cannot be read).
+int sm_count_current_device();
 
 // ---------------------------------------------------------------- host launchers
 // Each returns cudaGetLastError() after enqueuing on `stream`.

@@ -883,14 +883,10 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
 
 template <int D, int R>
 static cudaError_t launch_ex_t(const Problem& p, const CUtensorMap& gk, const CUtensorMap& gv, cudaStream_t st) {
-  static bool configured = false;
+  static PerDeviceFlag configured;
   const size_t smem = ExSmem<D, R>::total;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(exact_residual_kernel<D, R>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e = set_max_dynamic_smem(configured, reinterpret_cast<const void*>(exact_residual_kernel<D, R>), smem);
+  if (e != cudaSuccess) return e;
   dim3 grid((p.max_slices + kExGroups - 1) / kExGroups, p.n_q_heads, p.batch);
   return launch_pdl(exact_residual_kernel<D, R>, grid, dim3(kExThreads), smem, st, p);
 }
@@ -898,14 +894,11 @@ static cudaError_t launch_ex_t(const Problem& p, const CUtensorMap& gk, const CU
 template <int D, int R>
 static cudaError_t launch_ex_stream_t(const Problem& p, const CUtensorMap& gk, const CUtensorMap& gv, int n_ctas,
                                       cudaStream_t st) {
-  static bool configured = false;
+  static PerDeviceFlag configured;
   const size_t smem = ExStreamSmem<D, R>::total;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(exact_residual_stream_kernel<D, R>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e =
+      set_max_dynamic_smem(configured, reinterpret_cast<const void*>(exact_residual_stream_kernel<D, R>), smem);
+  if (e != cudaSuccess) return e;
   return launch_pdl(exact_residual_stream_kernel<D, R>, dim3(n_ctas), dim3(kExStreamThreads), smem, st, gk, gv, p);
 }
 

@@ -305,13 +305,10 @@ static size_t score_smem_bytes(int D) {
 
 template <int D>
 static cudaError_t launch_score_t(const Problem& p, const CUtensorMap& tm, int n_sm, cudaStream_t st) {
-  static bool configured = false;   // attribute is per function; cheap to set once
+  static PerDeviceFlag configured;
   const size_t smem = score_smem_bytes(D);
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(score_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e = set_max_dynamic_smem(configured, reinterpret_cast<const void*>(score_kernel<D>), smem);
+  if (e != cudaSuccess) return e;
   return launch_pdl(score_kernel<D>, dim3(n_sm), dim3(kScoreThreads), smem, st, tm, p);
 }
 

@@ -347,13 +347,10 @@ cudaError_t launch_select(const Problem& p, int max_mid, int n_sm, cudaStream_t 
     csize /= 2;
   const int n_tasks = p.with_phi ? rows + p.n_kv_heads : 0;
   const int feat_clusters = (n_tasks + csize - 1) / csize;
-  static bool configured = false;
+  static PerDeviceFlag configured;
   constexpr size_t smem = sizeof(unsigned) * kSelChunk;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e = set_max_dynamic_smem(configured, reinterpret_cast<const void*>(select_kernel), smem);
+  if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(csize, rows + feat_clusters, 1);
   cfg.blockDim = dim3(kSelThreads);

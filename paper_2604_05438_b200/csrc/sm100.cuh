@@ -47,10 +47,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // the CTA has raised *abort_flag (a shared-memory word); a thread that gives up on
 // its own raises the flag, so that every role of the CTA leaves its loop and the
 // CTA can tear down in an orderly way instead of hanging.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                uint32_t max_polls) {
   // pure polling first (a sleeping waiter wakes up late, and the hand-offs of a pipeline
   // add those delays up); back off only when the wait is clearly not a normal one
-  for (uint32_t i = 0; i < kWaitPolls; ++i) {
+  for (uint32_t i = 0; i < max_polls; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u) {
       if (*abort_flag) return false;
@@ -59,6 +60,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   }
   *abort_flag = 1;
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limit(bar, parity, abort_flag, kWaitPolls);
 }
 
 // Programmatic dependent launch: a kernel launched with the programmatic-serialization

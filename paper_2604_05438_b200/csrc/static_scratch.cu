@@ -9,8 +9,9 @@
 
 namespace {
 
-// Scratch shared by every call on a device.  Each GPU context that loads the library
-// holds these bytes until the process exits.
+// Scratch shared by every call on a device.  The array is part of this library's device
+// code: each GPU on which the CUDA runtime loads that code (at the latest on the first
+// call of the entry point below on that GPU) holds these bytes until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[TKPHI_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
@@ -65,9 +66,31 @@ tkphi_status tkphi_build_summaries_static(const tkphi_kv_desc* kv, const tkphi_p
     snprintf(g_static_err, sizeof(g_static_err), "looking up the built-in scratch: %s", cudaGetErrorString(e));
     return TKPHI_ERR_CUDA;
   }
-  // The build clears the counters it needs at the head of the scratch on the stream
-  // before its kernel runs, so whatever the previous call left there does not matter.
+  // Nothing in the scratch has to be cleared between calls: the build kernel sets the
+  // status word at its head itself and overwrites every partial sum before one is read.
   tkphi_status st = tkphi_build_summaries(kv, phi, S, u, scratch, (size_t)TKPHI_STATIC_SCRATCH_BYTES, cuda_stream);
+  if (st != TKPHI_OK) snprintf(g_static_err, sizeof(g_static_err), "%s", tkphi_last_error());
+  return st;
+}
+
+tkphi_status tkphi_static_device_status(void* cuda_stream, int32_t* status_out) {
+  g_static_err[0] = 0;
+  if (!status_out) {
+    snprintf(g_static_err, sizeof(g_static_err), "status_out is NULL");
+    return TKPHI_ERR_INVALID_ARG;
+  }
+  int dev = -1;
+  void* scratch = nullptr;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    scratch = g_scratch_addr[dev];
+  }
+  if (!scratch) {
+    snprintf(g_static_err, sizeof(g_static_err), "no tkphi_build_summaries_static call has been made on this device");
+    return TKPHI_ERR_INVALID_ARG;
+  }
+  // the status word is the first word of the scratch, as in a caller-provided workspace
+  tkphi_status st = tkphi_device_status(scratch, cuda_stream, status_out);
   if (st != TKPHI_OK) snprintf(g_static_err, sizeof(g_static_err), "%s", tkphi_last_error());
   return st;
 }

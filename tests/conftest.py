@@ -26,3 +26,19 @@ def read_golden(name="paper_values.txt"):
 @pytest.fixture(scope="session")
 def golden():
     return read_golden()
+
+
+@pytest.fixture(autouse=True)
+def parity_stats(request, capsys):
+    """GPU tests: one JSON line per test with the worst errors its parity helpers saw."""
+    if request.node.get_closest_marker("gpu") is None:
+        yield
+        return
+    import json
+
+    import parity_utils as PU
+    PU.STATS.clear()
+    yield
+    if PU.STATS:
+        with capsys.disabled():
+            print("\nPARITY " + json.dumps({"test": request.node.nodeid, "worst": PU.STATS}, sort_keys=True))

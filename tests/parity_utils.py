@@ -16,9 +16,21 @@ from workloads import LayerInputs, PhiParams, WorkloadConfig
 Y_TOL = 2e-3          # max_j |y_hat - y| / max_j |y| per output vector
 SU_TOL = 1e-3         # max |S_hat - S| / max |S| per head (same for u)
 TIE_TOL = 1e-5        # index sets may differ only where |s_i - tau| <= TIE_TOL * max(|tau|, 1)
-LOGZ_TOL = 2e-3       # absolute, on log Z_hat_R
+RESID_TOL = 2e-3      # residual terms, relative to the unsubtracted feature mass phi_q.u_M (see check_residual)
+DIR_MIN_LEFT = 0.005  # the residual direction is compared whenever more than this share of the mass is left
 ME_TOL = 1e-4         # absolute, on the exact-branch max score
 FP32_TINY = 1.2e-38   # below the smallest normal fp32 a summary entry is not representable
+
+# Worst errors seen by the helpers below since the last reset, by name; the GPU test modules print
+# them as one JSON line per test (conftest.py).
+STATS: dict = {}
+
+
+def note(name: str, value: float) -> float:
+    value = float(value)
+    if not (STATS.get(name, -math.inf) >= value):
+        STATS[name] = value
+    return value
 
 
 def max_rel(a, b) -> float:
@@ -94,9 +106,38 @@ def gpu_decode(gl: GpuLayer, q: torch.Tensor, topk: np.ndarray, S=None, u=None, 
 
 def seq_arrays(inp: LayerInputs, b: int, kvh: int):
     lo, hi = int(inp.cu_seqlens[b]), int(inp.cu_seqlens[b + 1])
-    K = inp.k[kvh, lo:hi].double().numpy()
-    V = inp.v[kvh, lo:hi].double().numpy()
+    K = inp.k[kvh, lo:hi].cpu().double().numpy()
+    V = inp.v[kvh, lo:hi].cpu().double().numpy()
     return K, V
+
+
+def check_residual(dbg_row, res, res_nosub, where) -> None:
+    """Residual terms of one query head against the oracle.
+
+    dbg_row: the library's debug row ([2] log Z_hat_R, [4:] nu_hat_R / Z_hat_R); res: the oracle's
+    result; res_nosub: the oracle's result with the subtraction skipped, whose log_Zhat_R is the
+    unsubtracted feature mass log(phi_q . u_M).
+
+    Z_hat_R = phi_q.u_M - sum_i z_i and nu_hat_R = S_M phi_q - sum_i z_i v_i are differences (Eq.
+    subtraction): rounding errors of the two sides do not shrink with the difference, so every
+    error is bounded relative to the unsubtracted mass phi_q.u_M.  With `left` the share of that
+    mass the subtraction leaves, the share itself is held to RESID_TOL, log Z_hat_R to
+    RESID_TOL / left, and the direction nu_hat_R / Z_hat_R to RESID_TOL / left of its largest entry
+    (both whenever left > DIR_MIN_LEFT; below that nothing but the share is meaningful).
+    """
+    log_ZM = res_nosub.log_Zhat_R
+    if not math.isfinite(log_ZM):
+        return                                   # no feature mass at all (zero summaries)
+    left = 0.0 if res.clamped else math.exp(res.log_Zhat_R - log_ZM)
+    got = math.exp(dbg_row[2] - log_ZM) if math.isfinite(dbg_row[2]) else 0.0   # -inf: clamped away
+    e_share = note("resid_share_abs_err", abs(got - left))
+    assert e_share <= RESID_TOL, (where, dbg_row[2], res.log_Zhat_R, left)
+    if left > DIR_MIN_LEFT:
+        e_log = note("resid_logz_err_x_left", abs(dbg_row[2] - res.log_Zhat_R) * left)
+        e_dir = note("resid_dir_err_x_left", max_rel(dbg_row[4:], res.y_R_hat) * left)
+        note("resid_min_left_checked", -left)
+        assert e_log <= RESID_TOL, (where, dbg_row[2], res.log_Zhat_R, left)
+        assert e_dir <= RESID_TOL, (where, e_dir, left)
 
 
 def check_selection(q64, K, n_sink, n_tail, topk, got_idx_row) -> np.ndarray:
@@ -118,14 +159,15 @@ def check_selection(q64, K, n_sink, n_tail, topk, got_idx_row) -> np.ndarray:
     return got
 
 
-def calibrate_visible_shift(cfg, inp: LayerInputs, phi: PhiParams, frac: float, n_probe: int = 4) -> torch.Tensor:
+def calibrate_visible_shift(cfg, inp: LayerInputs, phi: PhiParams, frac: float, n_probe: int = 4,
+                            kv_heads=None, b: int = 0) -> torch.Tensor:
     """Per-KV-head shift of b_k that puts median(log Z_hat_R - log Z_R) at zero
-    (computed with the oracle on a few queries of sequence 0)."""
+    (computed with the oracle on a few queries of sequence b; heads not in `kv_heads` keep 0)."""
     Hkv, G = cfg.n_kv_heads, cfg.group
     shifts = torch.zeros(Hkv)
-    b = 0
     topk = int(inp.topk(frac)[b])
-    for kvh in range(Hkv):
+    phi = phi.to("cpu")
+    for kvh in (range(Hkv) if kv_heads is None else kv_heads):
         K, V = seq_arrays(inp, b, kvh)
         S, u = O.build_summaries(K, V, phi.w_k[kvh].double().numpy(), phi.b_k[kvh].double().numpy(),
                                  phi.gamma_k, inp.n_sink, inp.n_tail)
@@ -133,7 +175,7 @@ def calibrate_visible_shift(cfg, inp: LayerInputs, phi: PhiParams, frac: float, 
         for n in range(n_probe):
             hq = kvh * G + (n % G)
             step = n // G % inp.q.shape[0]
-            q64 = inp.q[step, b, hq].double().numpy()
+            q64 = inp.q[step, b, hq].cpu().double().numpy()
             res = O.topkphi_attention(q64, K, V, inp.n_sink, inp.n_tail, topk,
                                       phi.w_q[hq].double().numpy(), phi.b_q[hq].double().numpy(), phi.gamma_q,
                                       phi.w_k[kvh].double().numpy(), phi.b_k[kvh].double().numpy(), phi.gamma_k,

@@ -60,6 +60,16 @@ def test_invalid_arguments_are_rejected_before_any_launch(lib):
     for bad in (dict(n_q=7), dict(n_sink=-1), dict(k=0), dict(k=0x1008), dict(st=60), dict(st=68)):
         dd, _c = _desc([0, 100], **bad)
         assert _decode(lib, dd, [1]) == -1, bad
+    # KV heads that share memory: a zero head stride, a head stride shorter than a head's rows
+    # (head-major) with a token stride too short to hold every head (token-major)
+    for bad in (dict(sh=0), dict(sh=64 * 50), dict(sh=64, st=64), dict(sh=32, st=128)):
+        dd, _c = _desc([0, 100], **bad)
+        assert _decode(lib, dd, [1]) == -1 and b"overlap" in lib.tkphi_last_error(), bad
+    for good in (dict(sh=64 * 100), dict(sh=64 * 100 + 8), dict(sh=64, st=128), dict(sh=72, st=144)):
+        dd, _c = _desc([0, 100], **good)
+        assert _decode(lib, dd, [1], ws=0) == -3, good       # passes validation, stops at the NULL workspace
+    dd, _c = _desc([0, 100], n_q=4, n_kv=1, sh=0)
+    assert _decode(lib, dd, [1], ws=0) == -3                 # one head: its stride is never used
     dd, _c = _desc([0, 100], n_q=18, n_kv=2)
     assert _decode(lib, dd, [1]) == -2                       # group of 9
     dd, _c = _desc([0, 100, 100])

@@ -282,6 +282,20 @@ def test_exact_sub_recovers_full_attention(golden):
     assert err < 1e-13
 
 
+def test_rel_l1_hand_computed_cases(golden):
+    # Sec. 6, metric definition: ||y_hat - y||_1 / (||y||_1 + eps), eps from the paper.
+    eps = golden["rel_l1_eps"]
+    assert eps == 1e-12
+    # |1.5-1| + |-2-(-2)| + |2-4| = 2.5 over |1| + |-2| + |4| = 7: a dropped abs, a squared norm
+    # or the hat vector in the denominator (5.5) all give another number
+    assert O.rel_l1([1.5, -2.0, 2.0], [1.0, -2.0, 4.0]) == pytest.approx(2.5 / (7.0 + eps), rel=1e-15)
+    assert O.rel_l1([1.0, -2.0, 4.0], [1.5, -2.0, 2.0]) == pytest.approx(2.5 / (5.5 + eps), rel=1e-15)
+    # a zero reference: the quotient is finite only because of eps, and eps is what the golden file says
+    assert O.rel_l1([3e-12, 0.0, -1e-12], [0.0, 0.0, 0.0]) == pytest.approx(4e-12 / eps, rel=1e-12)
+    assert O.rel_l1([3e-12, 0.0, -1e-12], [0.0, 0.0, 0.0], eps=eps) == O.rel_l1([3e-12, 0.0, -1e-12], [0.0, 0.0, 0.0])
+    assert O.rel_l1([0.25, 0.5], [0.25, 0.5]) == 0.0
+
+
 def test_reassociated_form_equals_literal():
     p = _rand_problem(15)
     res = _run(p, 7)

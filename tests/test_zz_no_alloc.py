@@ -35,6 +35,7 @@ def _both(cfg, seed, seq_lens):
     u = torch.full((B, Hkv, r), float("nan"), device=gl.dev)
     T.build_summaries_static(gl.kv, gl.maps, S, u)        # built-in scratch, no allocation inside
     torch.cuda.synchronize()
+    assert T.static_device_status() == 0                  # no bounded wait of the build kernel ran out
     return S_ref.cpu().numpy(), u_ref.cpu().numpy(), S.cpu().numpy(), u.cpu().numpy()
 
 
@@ -46,6 +47,27 @@ def test_static_scratch_build_matches_workspace_build_twice():
         assert PU.max_rel(S, S_ref) <= PU.SU_TOL and PU.max_rel(u, u_ref) <= PU.SU_TOL
         # same kernel, same summation order: in fact identical
         assert np.array_equal(S, S_ref) and np.array_equal(u, u_ref)
+
+
+def test_static_scratch_call_leaves_free_device_memory_unchanged():
+    # after one warm call (which loads the library's device code, the scratch array with it, and looks
+    # up its address) a further call must not take any device memory: not from the driver, not from
+    # torch's pool
+    import paper_2604_05438_b200 as T
+    cfg = dataclasses.replace(CONFIGS["c1_1b_4k"], n_q_heads=8, n_kv_heads=2)
+    inp = make_layer_inputs(cfg, 23, seq_lens=[2000], n_steps=1)
+    gl = PU.to_gpu(cfg, inp, make_phi_params(cfg, 23))
+    S = torch.empty(1, cfg.n_kv_heads, cfg.head_dim, cfg.n_feat, device=gl.dev)
+    u = torch.empty(1, cfg.n_kv_heads, cfg.n_feat, device=gl.dev)
+    T.build_summaries_static(gl.kv, gl.maps, S, u)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    reserved0 = torch.cuda.memory_reserved()
+    T.build_summaries_static(gl.kv, gl.maps, S, u)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and torch.cuda.memory_reserved() == reserved0
+    assert T.static_device_status() == 0
 
 
 def test_static_scratch_rejects_oversized_problems():

@@ -10,6 +10,7 @@ from .synthetic import (  # noqa: F401
     WorkloadConfig,
     LayerInputs,
     PhiParams,
+    draw_seq_lens,
     make_layer_inputs,
     make_phi_params,
     budget_to_topk,

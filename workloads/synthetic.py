@@ -154,6 +154,15 @@ def make_phi_params(cfg: WorkloadConfig, seed: int, kind: str = "baseline",
                      w_k.float().contiguous(), b_k.float().contiguous(), gq, gk, kind)
 
 
+def draw_seq_lens(cfg: WorkloadConfig, seed: int) -> List[int]:
+    """Prefill lengths of the workload's sequences: uniform in [seq_len_min, seq_len] for ragged
+    workloads (the same for every layer of a seed), else seq_len for all."""
+    if cfg.seq_len_min is None:
+        return [cfg.seq_len] * cfg.batch
+    gl = np.random.default_rng(seed * 7 + 3)
+    return [int(x) for x in gl.integers(cfg.seq_len_min, cfg.seq_len + 1, size=cfg.batch)]
+
+
 def make_layer_inputs(cfg: WorkloadConfig, seed: int, layer: int = 0, device="cpu",
                       seq_lens: Optional[List[int]] = None,
                       n_steps: Optional[int] = None) -> LayerInputs:
@@ -169,13 +178,9 @@ def make_layer_inputs(cfg: WorkloadConfig, seed: int, layer: int = 0, device="cp
     ones); ragged configs draw lengths uniformly in [seq_len_min, seq_len].
     """
     g = _gen(seed * 1000003 + layer * 101 + 1, device)
-    gl = np.random.default_rng(seed * 7 + 3)          # lengths: same for every layer
     B, Hq, Hkv, d = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     if seq_lens is None:
-        if cfg.seq_len_min is not None:
-            seq_lens = [int(x) for x in gl.integers(cfg.seq_len_min, cfg.seq_len + 1, size=B)]
-        else:
-            seq_lens = [cfg.seq_len] * B
+        seq_lens = draw_seq_lens(cfg, seed)
     B = len(seq_lens)
     steps = cfg.n_steps if n_steps is None else n_steps
     cu = np.zeros(B + 1, dtype=np.int64)
