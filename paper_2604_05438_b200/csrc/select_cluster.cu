@@ -7,32 +7,16 @@
 // (CTA, round, warp, step, lane) order is index order.  For sequences of up to 131072
 // mid-region keys every CTA keeps its 16384 order-preserving score keys in shared memory
 // and the row is read from L2 exactly once (longer rows, up to 2,097,152 keys, are read twice
-// and the shared memory holds per-round bit masks instead).
-//
-// The exact K-th largest key is found by histogram selection over WINDOWS of the 32-bit
-// order-preserving key: a window (lo, shift) maps a key >= lo to bin min((key - lo) >> shift,
-// 4095), which is monotone in the key, so counting from the top bin down to the bin where
-// the count reaches K brackets the threshold exactly whatever the window is.  The first
-// window is placed by a sample: every CTA of the cluster reads the same 2048 strided scores of
-// the row and takes, from a coarse histogram of them, a lower edge that lies below the K-th
-// largest score with high probability and an upper edge at the sample's maximum.  Keys below
-// the window (about 97% of a row at a 1% budget) cost no shared-memory atomic, and the bins
-// that are hit spread evenly, so the atomics neither collide nor leave a crowded threshold
-// bin: it holds a handful of keys instead of thousands.  When the sample misleads (the
-// threshold lies below the window, or in the clamped top bin) the count says so and the next
-// window covers exactly the range that is left; windows shrink by a factor of at least 2048
-// per level, so a few levels resolve any input, exact ties included.
-//
-// Every CTA builds a local histogram in shared memory and adds its non-zero bins into the
-// accumulator of every CTA through distributed shared memory; every CTA then walks its own copy.
-// A threshold bin of at most 512 keys is resolved directly: its (key, position) pairs are
-// gathered into every CTA and each thread ranks one of them (higher key first, lower position
-// first among equal keys).  Positions above the threshold, and as many threshold ties as are
-// still needed in index order, are then written straight to their slot of the ascending index
-// list: the per-thread bit masks are transposed inside each warp so that thread order is index
-// order, and offsets come from one block scan and per-CTA totals exchanged through distributed
-// shared memory.  CTAs of a cluster only meet at hardware cluster barriers (no flag spinning,
-// no global scratch, nothing to clear between calls).
+// and the shared memory holds per-round bit masks instead) (the loops over a thread's 32 keys stay rolled:
+// straight-line code that runs once is bound by instruction fetch, not by its work).  The exact K-th largest key is found by radix
+// selection over 12 + 10 + 10 bits: every CTA builds a local histogram in shared memory
+// and adds its non-zero bins into the accumulator of every CTA through distributed shared
+// memory; every CTA then walks its own copy of the accumulator.  Positions above the
+// threshold, and as many threshold ties as are still needed in index order, are then
+// written straight to their slot of the ascending index list: the per-thread bit masks
+// are transposed inside each warp so that thread order is index order, and offsets come
+// from one block scan and per-CTA totals exchanged through distributed shared memory.  CTAs of a cluster only meet at hardware cluster barriers
+// (no flag spinning, no global scratch, nothing to clear between calls).
 //
 // Extra clusters of the same launch do the work that depends only on the call's inputs
 // (query-side features, W_k operand split), off the critical path.
@@ -51,40 +35,34 @@ constexpr int kSelPer = 32;                              // scores per thread an
 constexpr int kSelChunk = kSelThreads * kSelPer;         // 16384 scores per CTA and round
 constexpr int kSelCluster = 8;                            // largest cluster; the launch picks 1, 2, 4 or 8
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kSamplePer = 4;                            // sampled scores per thread
-constexpr int kSampleMax = kSelThreads * kSamplePer;     // scores of a row that place the first window
-constexpr int kCandCap = kSelThreads;                    // a threshold bin of up to this many keys is ranked directly
-constexpr int kSelLevels = 8;                            // windows per row, at most (five suffice for any input)
+constexpr int kRefBins = 1024;                           // two refinement digits of 10 bits
 
 struct SelShared {
-  unsigned hist[kHistBins];      // local histogram of the current window
-  unsigned acc[kHistBins];       // the cluster's histogram (every CTA receives every CTA's bins)
-  unsigned cand_key[kCandCap];   // keys of the threshold bin, gathered from the whole cluster
-  int cand_pos[kCandCap];        // their mid-region positions
-  unsigned selw[kSelThreads];    // resident mode: selection bits that the direct ranking decided
-  unsigned cand_n;               // entries of the candidate list
-  unsigned wmax[kSelWarps];
+  unsigned hist[kHistBins];      // local 12-bit histogram
+  unsigned acc[kHistBins];       // the cluster's 12-bit histogram (every CTA receives every CTA's bins)
+  unsigned h1[kRefBins];         // local refinement histogram
+  unsigned acc1[kRefBins];       // the cluster's histogram of refinement digit 1
+  unsigned acc2[kRefBins];       // ... of refinement digit 2
   int scratch[40];
-  int res[4];                    // result of a histogram walk: bin (-1: not reached), count above it, count in it, total
+  int res[4];                    // result of a histogram walk: digit, count above it, count in it
   int tot[2 * kSelCluster];      // per CTA: selected-for-sure count, tie count
   int wdef[kSelWarps], wtie[kSelWarps];
 };
 
-// Walks the kHistBins-bin histogram h from the top and finds the bin at which the cumulative
-// count reaches `need`; res = {bin, count above it, count in it, count of all bins}, bin = -1
-// when the histogram holds fewer than `need` entries.  All 512 threads of the CTA call it.
+// Walks an n-bin histogram (n = NB, a multiple of 512) from the top and finds the bin at
+// which the cumulative count reaches `need`; res = {bin, count above it, count in it}.
+// All 512 threads of the CTA call it.
+template <int NB>
 __device__ void walk_from_top(const unsigned* h, int need, int* res, int* scratch) {
-  constexpr int BPT = kHistBins / kSelThreads;
+  constexpr int BPT = NB / kSelThreads;
   const int tid = threadIdx.x;
   unsigned loc[BPT];
   int lsum = 0;
 #pragma unroll
   for (int i = 0; i < BPT; ++i) { loc[i] = h[tid * BPT + i]; lsum += (int)loc[i]; }
-  if (tid == 0) res[0] = -1;                               // (ordered before the finder's write by the scan's barriers)
   int total;
   const int excl = block_exclusive_scan(lsum, scratch, &total);
   const int above = total - excl - lsum;                   // elements in bins above this thread's range
-  if (tid == 0) res[3] = total;
   if (above < need && need <= above + lsum) {
     int cum = above;
 #pragma unroll
@@ -110,11 +88,6 @@ __device__ __forceinline__ unsigned warp_transpose32(unsigned x, int lane) {
   return x;
 }
 
-// smallest s with 2^s >= x (x >= 1)
-__device__ __forceinline__ int ceil_log2_u64(unsigned long long x) {
-  return x <= 1 ? 0 : 64 - __clzll((long long)(x - 1));
-}
-
 __global__ void __launch_bounds__(kSelThreads, 2)
 select_kernel(const Problem p, const int n_rows, const int csize) {
   __shared__ SelShared sm;
@@ -135,8 +108,9 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
     }
     return;
   }
-  // Everything up to the wait reads only the call's inputs (sequence lengths, budgets) and
-  // this CTA's shared memory, so it overlaps the scoring kernel's run.
+  // Everything up to the wait reads only the call's inputs (sequence lengths, budgets) and this
+  // CTA's shared memory, so it overlaps the scoring kernel's run: the first loads of the score
+  // row are issued 1.5 us earlier than with the wait at the top.
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int row = blockIdx.y, b = row / p.n_q_heads, hq = row % p.n_q_heads;
@@ -147,11 +121,10 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
   const int n_chunks = (n_mid + kSelChunk - 1) / kSelChunk;
   const int rounds = (n_chunks + csize - 1) / csize;       // per CTA
   const bool resident = rounds == 1;                       // the keys stay in shared memory
+  const unsigned low_mask = (1u << kLowBits) - 1u;
   for (int i = tid; i < kHistBins; i += kSelThreads) { sm.hist[i] = 0; sm.acc[i] = 0; }
-  sm.selw[tid] = 0;
-  if (tid == 0) sm.cand_n = 0;
+  for (int i = tid; i < kRefBins; i += kSelThreads) { sm.h1[i] = 0; sm.acc1[i] = 0; sm.acc2[i] = 0; }
   pdl_wait();                                              // score rows and workspace of the predecessors
-
   int* out = p.idx + (size_t)row * p.topk_max;
   int* out2 = p.idx_out ? p.idx_out + (size_t)row * p.topk_max : nullptr;
   if (out2 && rank == 0)
@@ -181,99 +154,42 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
   auto key_at = [&](int k, int i) -> unsigned {            // key i of round k (valid positions only)
     return resident ? keys[i * kSelThreads] : ordered_key(__ldcg(srow + round_base(k) + i * 32));
   };
-  // adds the non-zero bins of the local histogram into the accumulator of every CTA
-  auto push_all = [&]() {
-    for (int i = tid; i < kHistBins; i += kSelThreads) {
-      const unsigned c = sm.hist[i];
-      if (c)
-        for (int r = 0; r < csize; ++r) atomicAdd(cluster.map_shared_rank(sm.acc, r) + i, c);
+  // adds the non-zero bins of a local histogram into the accumulator of every CTA
+  auto push_all = [&](unsigned* local, unsigned* accum, int n_bins, bool clear) {
+    for (int i = tid; i < n_bins; i += kSelThreads) {
+      const unsigned c = local[i];
+      if (c) {
+        for (int r = 0; r < csize; ++r) atomicAdd(cluster.map_shared_rank(accum, r) + i, c);
+        if (clear) local[i] = 0;
+      }
     }
   };
 
-  // ---- the row's sample (the same positions in every CTA of the cluster) and, in resident
-  // mode, this thread's 32 scores: all loads are issued before the first one is used
-  const int m_s = n_mid < kSampleMax ? n_mid : kSampleMax;
-  int r_s;                                                 // rank, in the sample, of the first window's lower edge
-  {
-    const float mp = (float)m_s * (float)K / (float)n_mid;
-    r_s = (int)ceilf(mp + 4.f * sqrtf(mp) + 4.f);          // the expected rank of the threshold plus four deviations
-  }
-  const bool sampled = r_s < m_s;                          // otherwise the first window is the whole key range
-  unsigned skey[kSamplePer];
-#pragma unroll
-  for (int e = 0; e < kSamplePer; ++e) {
-    const int j = tid + e * kSelThreads;
-    skey[e] = (sampled && j < m_s) ? ordered_key(__ldcg(srow + (long long)j * n_mid / m_s)) : 0u;
-  }
-  unsigned kr0[kSelPer];
-  unsigned vmask0 = 0;                                     // validity mask of the resident round
-  if (resident) vmask0 = load_regs(0, kr0);
+  // ---- 12-bit histogram of the row, replicated in every CTA (the histograms were cleared before the wait)
   __syncthreads();
-
-  unsigned win_lo = 0;                                     // first window: keys >= win_lo, bins of 2^win_shift keys
-  int win_shift = kLowBits;
-  if (sampled) {
-    unsigned smax = 0;
-#pragma unroll
-    for (int e = 0; e < kSamplePer; ++e)
-      if (tid + e * kSelThreads < m_s) {
-        atomicAdd(&sm.acc[skey[e] >> kLowBits], 1u);
-        smax = max(smax, skey[e]);
-      }
-    smax = __reduce_max_sync(0xffffffffu, smax);
-    if (lane == 0) sm.wmax[warp] = smax;
-    __syncthreads();
-    walk_from_top(sm.acc, r_s, sm.res, sm.scratch);        // r_s <= m_s: always found
-    const unsigned cb = (unsigned)sm.res[0];
-    unsigned cbmax = 0;
-#pragma unroll
-    for (int w = 0; w < kSelWarps; ++w) cbmax = max(cbmax, sm.wmax[w]);
-    cbmax >>= kLowBits;
-    win_lo = cb << kLowBits;
-    win_shift = kLowBits - kHistBits + ceil_log2_u64((unsigned long long)(cbmax - cb + 1));
-#pragma unroll
-    for (int e = 0; e < kSamplePer; ++e)
-      if (tid + e * kSelThreads < m_s) sm.acc[skey[e] >> kLowBits] = 0;   // the accumulator is clean again
-    __syncthreads();
-  }
-  cluster.barrier_arrive();                                // "my accumulator is cleared"; waited for below
-
-  // ---- histogram of the first window
+  cluster.barrier_arrive();                                // "my accumulators are cleared"; waited for below
+  unsigned vmask0 = 0;                                     // validity mask of the resident round
   for (int k = 0; k < rounds; ++k) {
-    unsigned vm = vmask0;
-    if (!resident) vm = load_regs(k, kr0);
+    unsigned kr[kSelPer];
+    const unsigned vm = load_regs(k, kr);
 #pragma unroll
     for (int i = 0; i < kSelPer; ++i) {
-      if (resident) keys[i * kSelThreads] = kr0[i];
-      if (((vm >> i) & 1u) && kr0[i] >= win_lo)
-        atomicAdd(&sm.hist[min((kr0[i] - win_lo) >> win_shift, (unsigned)(kHistBins - 1))], 1u);
+      if (resident) keys[i * kSelThreads] = kr[i];
+      if ((vm >> i) & 1u) atomicAdd(&sm.hist[kr[i] >> kLowBits], 1u);
     }
+    vmask0 = vm;
   }
   __syncthreads();
   cluster.barrier_wait();                                  // every accumulator of the cluster is cleared
-  push_all();
+  push_all(sm.hist, sm.acc, kHistBins, false);
   cluster.sync();
-  walk_from_top(sm.acc, K, sm.res, sm.scratch);
+  walk_from_top<kHistBins>(sm.acc, K, sm.res, sm.scratch);
+  const unsigned tb = (unsigned)sm.res[0];                 // threshold bin
+  const int need = K - sm.res[1];                          // keys to take inside it, 1 <= need <= n_cand
+  const int n_cand = sm.res[2];
+  const bool refine = need < n_cand;                       // the same in every CTA
 
-  // The threshold lies in the key range [r_lo, r_hi]: keys above it are selected for sure,
-  // `need` of the n_cand keys inside it are still to be taken.
-  unsigned r_lo, r_hi;
-  int need, n_cand;
-  if (sm.res[0] >= 0) {
-    const unsigned long long lo64 = (unsigned long long)win_lo + ((unsigned long long)sm.res[0] << win_shift);
-    const unsigned long long hi64 = sm.res[0] == kHistBins - 1 ? 0xffffffffull : lo64 + (1ull << win_shift) - 1;
-    r_lo = (unsigned)lo64;
-    r_hi = (unsigned)(hi64 < 0xffffffffull ? hi64 : 0xffffffffull);
-    need = K - sm.res[1];
-    n_cand = sm.res[2];
-  } else {                                                 // fewer than K keys in the window: the threshold lies below it
-    r_lo = 0;
-    r_hi = win_lo - 1;                                     // (win_lo > 0: a whole-range window holds every key)
-    need = K - sm.res[3];
-    n_cand = n_mid - sm.res[3];
-  }
-
-  // bit i of a "sure" mask: key i lies above the range; of a "cand" mask: inside it
+  // bit i of a "sure" mask: key i lies above the threshold bin; of a "cand" mask: inside it
   unsigned smask = 0, cmask = 0;                           // resident mode
   auto get_masks = [&](int k, unsigned* s_, unsigned* c_) {
     if (resident) { *s_ = smask; *c_ = cmask; }
@@ -287,109 +203,74 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
     unsigned s_ = 0, c_ = 0;
 #pragma unroll 4
     for (int i = 0; i < kSelPer; ++i) {
-      const unsigned key = keys[i * kSelThreads];
-      s_ |= (key > r_hi ? 1u : 0u) << i;
-      c_ |= ((key >= r_lo && key <= r_hi) ? 1u : 0u) << i;
+      const unsigned bin = keys[i * kSelThreads] >> kLowBits;
+      s_ |= (bin > tb ? 1u : 0u) << i;
+      c_ |= (bin == tb ? 1u : 0u) << i;
     }
     smask = s_ & vmask0; cmask = c_ & vmask0;
   } else {
     for (int k = 0; k < rounds; ++k) {
-      const unsigned vm = load_regs(k, kr0);
+      unsigned kr[kSelPer];
+      const unsigned vm = load_regs(k, kr);
       unsigned s_ = 0, c_ = 0;
 #pragma unroll
       for (int i = 0; i < kSelPer; ++i) {
-        s_ |= (kr0[i] > r_hi ? 1u : 0u) << i;
-        c_ |= ((kr0[i] >= r_lo && kr0[i] <= r_hi) ? 1u : 0u) << i;
+        const unsigned bin = kr[i] >> kLowBits;
+        s_ |= (bin > tb ? 1u : 0u) << i;
+        c_ |= (bin == tb ? 1u : 0u) << i;
       }
       put_masks(k, s_ & vm, c_ & vm);
     }
   }
 
-  // ---- resolve the threshold range.  Every decision below depends only on the cluster's
-  // histogram, so all CTAs of the cluster take the same path and meet at the same barriers.
-  int need_ties = n_cand;                                  // need == n_cand: the whole range is taken
-  for (int level = 0; level < kSelLevels && need < n_cand; ++level) {
-    if (n_cand <= kCandCap) {
-      // ---- direct ranking: every CTA gets every (key, position) of the range
-      for (int k = 0; k < rounds; ++k) {
-        unsigned s_, c_;
-        get_masks(k, &s_, &c_);
-        for (unsigned m = c_; m; m &= m - 1) {
-          const int i = __ffs(m) - 1;
-          const unsigned key = key_at(k, i);
-          const int pos = round_base(k) + i * 32;
-          for (int r = 0; r < csize; ++r) {
-            const unsigned slot = atomicAdd(cluster.map_shared_rank(&sm.cand_n, r), 1u);
-            if (slot < (unsigned)kCandCap) {
-              cluster.map_shared_rank(sm.cand_key, r)[slot] = key;
-              cluster.map_shared_rank(sm.cand_pos, r)[slot] = pos;
-            }
-          }
-        }
-      }
-      cluster.sync();
-      if (tid < n_cand) {
-        const unsigned mykey = sm.cand_key[tid];
-        const int mypos = sm.cand_pos[tid];
-        int better = 0;                                    // keys of the range that come before this one
-        for (int j = 0; j < n_cand; ++j) {
-          const unsigned kj = sm.cand_key[j];
-          better += (kj > mykey || (kj == mykey && sm.cand_pos[j] < mypos)) ? 1 : 0;
-        }
-        const int local = mypos - rank * rounds * kSelChunk;
-        if (better < need && local >= 0 && local < rounds * kSelChunk) {
-          const int k = local / kSelChunk, in = local % kSelChunk;
-          const int t = (in >> 10) * 32 + (in & 31), i = (in >> 5) & 31;
-          if (resident) atomicOr(&sm.selw[t], 1u << i);
-          else atomicOr(&keys_s[(2 * k) * kSelThreads + t], 1u << i);
-        }
-      }
-      __syncthreads();
-      if (resident) { smask |= sm.selw[tid]; cmask = 0; }
-      else
-        for (int k = 0; k < rounds; ++k) keys_s[(2 * k + 1) * kSelThreads + tid] = 0;
-      need_ties = 0;
-      break;
-    }
-    if (r_lo == r_hi) { need_ties = need; break; }         // one key value: exact ties, admitted in index order
-    // ---- next window: the whole range that is left, in 4096 bins
-    const int z_shift = max(0, ceil_log2_u64((unsigned long long)r_hi - r_lo + 1) - kHistBits);
-    for (int i = tid; i < kHistBins; i += kSelThreads) { sm.hist[i] = 0; sm.acc[i] = 0; }
-    __syncthreads();
-    cluster.sync();                                        // every accumulator of the cluster is cleared
+  unsigned tau_low = 0;
+  int need_ties = n_cand;
+  if (refine) {
+    // ---- digit 1: bits 19..10 of the key among the keys of the threshold bin
     for (int k = 0; k < rounds; ++k) {
       unsigned s_, c_;
       get_masks(k, &s_, &c_);
-      for (unsigned m = c_; m; m &= m - 1) atomicAdd(&sm.hist[(key_at(k, __ffs(m) - 1) - r_lo) >> z_shift], 1u);
+      for (unsigned m = c_; m; m &= m - 1) atomicAdd(&sm.h1[(key_at(k, __ffs(m) - 1) & low_mask) >> 10], 1u);
     }
     __syncthreads();
-    push_all();
+    push_all(sm.h1, sm.acc1, kRefBins, true);
     cluster.sync();
-    walk_from_top(sm.acc, need, sm.res, sm.scratch);       // need <= n_cand: always found
-    const unsigned long long lo64 = (unsigned long long)r_lo + ((unsigned long long)sm.res[0] << z_shift);
-    const unsigned long long hi64 = lo64 + (1ull << z_shift) - 1;
-    const unsigned n_lo = (unsigned)lo64, n_hi = hi64 < (unsigned long long)r_hi ? (unsigned)hi64 : r_hi;
+    walk_from_top<kRefBins>(sm.acc1, need, sm.res, sm.scratch);
+    const unsigned d1 = (unsigned)sm.res[0];
+    const int rem1 = need - sm.res[1];
+    __syncthreads();
+    // ---- digit 2: bits 9..0 among the keys whose digit 1 matches
     for (int k = 0; k < rounds; ++k) {
-      unsigned s_, c_, keep = 0;
+      unsigned s_, c_;
+      get_masks(k, &s_, &c_);
+      for (unsigned m = c_; m; m &= m - 1) {
+        const unsigned low = key_at(k, __ffs(m) - 1) & low_mask;
+        if ((low >> 10) == d1) atomicAdd(&sm.h1[low & (kRefBins - 1)], 1u);
+      }
+    }
+    __syncthreads();
+    push_all(sm.h1, sm.acc2, kRefBins, false);
+    cluster.sync();
+    walk_from_top<kRefBins>(sm.acc2, rem1, sm.res, sm.scratch);
+    tau_low = (d1 << 10) | (unsigned)sm.res[0];
+    need_ties = rem1 - sm.res[1];
+  }
+
+  // after this, "sure": keys above the exact threshold; "cand": keys equal to it (without
+  // refinement the whole threshold bin counts as tied: all of it is taken)
+  if (refine) {
+    for (int k = 0; k < rounds; ++k) {
+      unsigned s_, c_, tie = 0;
       get_masks(k, &s_, &c_);
       for (unsigned m = c_; m; m &= m - 1) {
         const int i = __ffs(m) - 1;
-        const unsigned key = key_at(k, i);
-        if (key > n_hi) s_ |= 1u << i;
-        else if (key >= n_lo) keep |= 1u << i;
+        const unsigned low = key_at(k, i) & low_mask;
+        if (low > tau_low) s_ |= 1u << i;
+        else if (low == tau_low) tie |= 1u << i;
       }
-      put_masks(k, s_, keep);
+      put_masks(k, s_, tie);
     }
-    need -= sm.res[1];
-    n_cand = sm.res[2];
-    r_lo = n_lo;
-    r_hi = n_hi;
-    need_ties = n_cand;                                    // (if the loop ends here, need == n_cand)
-    __syncthreads();                                       // sm.res is rewritten by the next walk
   }
-
-  // after this, "sure": keys above the exact threshold; "cand": keys equal to it, of which the
-  // first need_ties in index order are taken
 
   // ---- per-CTA totals, exchanged so that every CTA knows what the CTAs before it contribute
   {
