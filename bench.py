@@ -31,8 +31,6 @@ sys.path.insert(0, ROOT)
 
 from workloads import CONFIGS, make_layer_inputs, make_phi_params  # noqa: E402
 
-L2_BYTES = 126e6
-
 
 def _peaks():
     """(HBM GB/s, bf16 TFLOP/s burst, bf16 TFLOP/s sustained, "measured" | "fallback")."""
@@ -44,9 +42,9 @@ def _peaks():
     return 6650.0, 1590.0, 1400.0, "fallback"
 
 
-# DRAM bytes per launch of the scoring kernel from the committed ncu capture of this kernel
-# (profiles/); None once the kernel has changed since the capture.
-SCORE_KERNEL_NCU_TRAFFIC_BYTES = 268231936 + 3233792    # dram read + write, profiles/decode_kernels_c3_one_layer.md
+# DRAM bytes (read + write) of one launch of the scoring kernel, from an ncu capture of this kernel on the
+# workload below; set to None when the kernel changes, until the counters have been taken again.
+SCORE_KERNEL_NCU_TRAFFIC = {"config": "c3_3b_128k", "budget": 0.01, "bytes": 268231936 + 3233792}
 
 
 # --------------------------------------------------------------------------- clocks
@@ -116,6 +114,15 @@ def algorithmic_bytes(cfg, seq_lens, topk, n_layers):
     per_layer = key_stream + gather + su + weights
     return {"key_stream": key_stream * n_layers, "total": per_layer * n_layers,
             "key_stream_per_layer": key_stream}
+
+
+def workload_string(cfg, n_layers, N, budget, tmax, seq_lens=None):
+    """The same text in both arms, so that the two lines can be matched."""
+    s = (f"{cfg.name}: {n_layers} layers x {cfg.n_q_heads}q/{cfg.n_kv_heads}kv heads, d={cfg.head_dim}, "
+         f"r={cfg.n_feat}, N={N}, anchors {cfg.n_sink}+{cfg.n_tail}, budget {budget:g} (K<={tmax}), batch {cfg.batch}")
+    if seq_lens is not None and len(set(seq_lens)) > 1:
+        s += f", ragged lengths {min(seq_lens)}..{max(seq_lens)}"
+    return s
 
 
 def run_ours(args, rank, world, device):
@@ -236,9 +243,7 @@ def run_ours(args, rank, world, device):
         "value": ms * 1e3, "unit": "us/step", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 K/V, f32 accumulate", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: {n_layers} layers x {Hq}q/{Hkv}kv heads, d={d}, r={r}, N={N}, "
-                               f"anchors {cfg.n_sink}+{cfg.n_tail}, budget {args.budget:g} (K<={tmax}), batch {B}"
-                               + (f", ragged lengths {min(seq_lens)}..{max(seq_lens)}" if len(set(seq_lens)) > 1 else ""),
+        "config": {"workload": workload_string(cfg, n_layers, N, args.budget, tmax, seq_lens),
                    "l2": "inputs (K/V of all layers) exceed L2 by >100x; no flush needed",
                    "replicas": world, "seed": seed},
         "step_us": {"median": statistics.median(per_step) * 1e3, "min": min(per_step) * 1e3,
@@ -258,8 +263,12 @@ def run_ours(args, rank, world, device):
     if kt is not None:
         dom = kt["score"]
         a = ab["key_stream_per_layer"] / (dom["avg_ms"] * 1e-3) / 1e9
-        out["roofline"] = {"bound": "hbm", "kernel": "score_kernel", "achieved": a, "peak": peak,
-                           "unit": "GB/s", "frac": a / peak, "traffic": SCORE_KERNEL_NCU_TRAFFIC_BYTES,
+        t = SCORE_KERNEL_NCU_TRAFFIC
+        traffic = (t["bytes"] if t and t["config"] == args.config and abs(t["budget"] - args.budget) < 1e-9
+                   and not args.seq_len else None)
+        out["roofline"] = {"bound": "hbm", "kernel": "score_kernel", "scope": "score_kernel only (the whole step: "
+                           "hbm_frac_of_measured_peak)", "achieved": a, "peak": peak,
+                           "unit": "GB/s", "frac": a / peak, "traffic": traffic,
                            "peak_kind": peak_kind, "algorithmic_bytes_per_launch": ab["key_stream_per_layer"],
                            "avg_launch_us": dom["avg_ms"] * 1e3}
         out["kernels_us_per_launch"] = {k: v["avg_ms"] * 1e3 for k, v in kt.items()}
@@ -300,7 +309,7 @@ class OracleSample:
     Inputs and the prefill summaries are prepared once; `step(i)` times one decode query per
     sampled head and scales to a full step (all heads, all sequences, one layer)."""
 
-    def __init__(self, cfg, N, budget, n_heads, n_queries, seed=0):
+    def __init__(self, cfg, N, budget, n_heads, n_queries, seed=0, fixed_len=True):
         from oracle import tkphi_oracle as O
         self.O, self.cfg = O, cfg
         try:
@@ -308,7 +317,8 @@ class OracleSample:
             self.threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
         except Exception:
             self.threads = 1
-        self.inp = make_layer_inputs(cfg, seed, layer=0, seq_lens=[N] * cfg.batch, n_steps=n_queries)
+        self.inp = make_layer_inputs(cfg, seed, layer=0, seq_lens=[N] * cfg.batch if fixed_len else None,
+                                     n_steps=n_queries)
         self.phi = make_phi_params(cfg, seed)
         self.topk = int(self.inp.topk(budget)[0])
         G = cfg.group
@@ -344,23 +354,25 @@ def run_reference(args):
     n_layers = args.layers or cfg.n_layers
     N = args.seq_len or cfg.seq_len
     n_heads = 2
-    smp = OracleSample(cfg, N, args.budget, n_heads, n_queries=max(1, min(16, args.warmup + args.steps)))
+    smp = OracleSample(cfg, N, args.budget, n_heads, n_queries=max(1, min(16, args.warmup + args.steps)),
+                       fixed_len=bool(args.seq_len) or cfg.seq_len_min is None)
     vals = []
     for s in range(args.warmup + args.steps):
         dt, per_layer_s = smp.step(s)
         if s >= args.warmup:
             vals.append(per_layer_s * n_layers)
     us = statistics.mean(vals) * 1e6
-    tmax = int(math.floor(args.budget * (N - cfg.n_sink - cfg.n_tail) + 1e-9))
+    seq_lens = [smp.inp.seq_len(b) for b in range(smp.inp.batch)]
+    tmax = int(smp.inp.topk(args.budget).max())
+    scale = cfg.n_q_heads * cfg.batch * n_layers / n_heads
     sample = (f"{n_heads} of {cfg.n_q_heads} query heads of sequence 0 of one layer per step, full N={N}, "
               f"scaled by heads, {cfg.batch} sequence(s) and {n_layers} layers; summaries prebuilt")
     return {
         "impl": "reference", "metric": "Top-K+phi decode-step latency (us), 128K ctx", "value": us,
         "unit": "us/step", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3,
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: {n_layers} layers x {cfg.n_q_heads}q/{cfg.n_kv_heads}kv heads, "
-                               f"d={cfg.head_dim}, r={cfg.n_feat}, N={N}, anchors {cfg.n_sink}+{cfg.n_tail}, "
-                               f"budget {args.budget:g} (K={tmax}), batch {cfg.batch}"},
+        "config": {"workload": workload_string(cfg, n_layers, N, args.budget, tmax, seq_lens)},
+        "extrapolated": True, "scale_factor": scale,
         "cpu_baseline": {"value": us, "unit": "us/step", "cores": smp.threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -402,7 +414,8 @@ def main():
             cfg = CONFIGS[args.config]
             n_layers = args.layers or cfg.n_layers
             N = args.seq_len or cfg.seq_len
-            smp = OracleSample(cfg, N, args.budget, 8, n_queries=16)
+            smp = OracleSample(cfg, N, args.budget, 8, n_queries=16,
+                               fixed_len=bool(args.seq_len) or cfg.seq_len_min is None)
             dts, ests = zip(*[smp.step(i) for i in range(16)])
             out["cpu_baseline"] = {
                 "value": statistics.mean(ests) * n_layers * 1e6, "unit": "us/step", "cores": smp.threads,
