@@ -99,13 +99,25 @@ typedef struct {
 } tkphi_kv_desc;
 
 /* phi(x) = exp(W x + b - gamma ||x||^2); row-major fp32 parameters on the device; w_q and
- * w_k 16-byte aligned (as are S and u where a call takes them). */
+ * w_k 16-byte aligned (as are S and u where a call takes them).
+ *
+ * phi_k_cache (optional, NULL to leave out) is the cached-feature variant that Sec. 4.2
+ * names as a way to avoid recomputing the retrieved keys' feature maps at decode time:
+ * device fp32 [n_kv_heads][T_total][n_feat], T_total = cu_seqlens[batch], 16-byte aligned,
+ * owned by the caller.  tkphi_build_summaries, given a non-NULL pointer, also writes
+ * phi_k(k_i) of every mid-region token i of every sequence to row cu_seqlens[b] + i of each
+ * KV head (rows of anchor tokens are left untouched).  tkphi_decode_step, given a non-NULL
+ * pointer, takes the retrieved tokens' feature rows from it instead of recomputing them from
+ * the keys (Eq. subtraction is unchanged: the same phi_k(k_i) enter it); the rows must hold
+ * what the build wrote for the same cache, anchors and parameters (w_k, b_k and gamma_k are
+ * then not read by the decode step).  tkphi_topk_decode and the NoSub flag ignore it. */
 typedef struct {
   const float* w_q; /* [n_q_heads][n_feat][head_dim] */
   const float* b_q; /* [n_q_heads][n_feat] */
   const float* w_k; /* [n_kv_heads][n_feat][head_dim] */
   const float* b_k; /* [n_kv_heads][n_feat] */
   float gamma_q, gamma_k;
+  float* phi_k_cache; /* optional, [n_kv_heads][T_total][n_feat] */
 } tkphi_phi_desc;
 
 /*
@@ -249,7 +261,8 @@ enum {
   TKPHI_KERNEL_EXACT_RESIDUAL = 2,  /* exact branch, subtraction, residual, merge */
   TKPHI_KERNEL_BUILD = 3,           /* prefill summary build */
   TKPHI_KERNEL_MEMSET = 4,          /* clearing counters when there is nothing to score */
-  TKPHI_KERNEL_KINDS = 5
+  TKPHI_KERNEL_CACHED_Z = 5,        /* <phi_q, cached phi_k row> of the retrieved tokens (phi_k_cache given) */
+  TKPHI_KERNEL_KINDS = 6
 };
 void tkphi_kernel_timing_enable(int32_t on);
 tkphi_status tkphi_kernel_timing_read(float* ms_out, int32_t* count_out);

@@ -284,6 +284,23 @@ def topkphi_attention(q, K, V, n_sink, n_tail, topk, W_q, b_q, gamma_q, W_k, b_k
                                phi_log(q, W_q, b_q, gamma_q), Phi_ret, subtract=subtract)
 
 
+def topkphi_attention_cached(q, K, V, n_sink, n_tail, topk, W_q, b_q, gamma_q, Phi_cache, S, u,
+                             retrieved=None, subtract: bool = True) -> TopKPhiResult:
+    """Top-K+phi with cached key features (Sec. 4.2 notes that a cached implementation avoids the
+    decode-time recompute): Phi_cache[i] = phi_k(k_i) for every mid-region row i, as stored when
+    the summaries (S, u) were built.  Eq. (subtraction) takes the retrieved rows of the cache as
+    they are; nothing else changes.
+    """
+    K = np.asarray(K, F64)
+    if retrieved is None:
+        retrieved = select_topk(q, K, n_sink, n_tail, topk)
+    retrieved = np.asarray(retrieved, np.int64)
+    Phi_cache = np.asarray(Phi_cache, F64)
+    Phi_ret = Phi_cache[retrieved] if retrieved.size else np.zeros((0, Phi_cache.shape[1]), F64)
+    return merge_from_features(q, K, V, n_sink, n_tail, retrieved, S, u,
+                               phi_log(q, W_q, b_q, gamma_q), Phi_ret, subtract=subtract)
+
+
 def topkphi_attention_generated(q, K_all, V_all, n_prefill: int, n_sink, n_tail, topk,
                                 W_q, b_q, gamma_q, W_k, b_k, gamma_k, S=None, u=None, retrieved=None):
     """Decode with already generated tokens kept exact (Sec. 4.3, Eq. implemented_decode):

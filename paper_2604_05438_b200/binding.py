@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "tkphi_selftest_timeout",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
-KERNEL_KINDS = ("score", "select", "exact_residual", "build", "memset")
+KERNEL_KINDS = ("score", "select", "exact_residual", "build", "memset", "cached_z")
 ERR_TIMEOUT = -5
 
 
@@ -44,7 +44,7 @@ class _KvDesc(C.Structure):
 
 class _PhiDesc(C.Structure):
     _fields_ = [("w_q", C.c_void_p), ("b_q", C.c_void_p), ("w_k", C.c_void_p), ("b_k", C.c_void_p),
-                ("gamma_q", C.c_float), ("gamma_k", C.c_float)]
+                ("gamma_q", C.c_float), ("gamma_k", C.c_float), ("phi_k_cache", C.c_void_p)]
 
 
 def library_path() -> str:
@@ -151,12 +151,17 @@ class PhiMaps:
     b_k: torch.Tensor
     gamma_q: float
     gamma_k: float
+    phi_k_cache: Optional[torch.Tensor] = None   # optional fp32 [n_kv_heads][T_total][n_feat]: written by the build, read by decode_step
 
     def desc(self) -> _PhiDesc:
         for t in (self.w_q, self.b_q, self.w_k, self.b_k):
             assert t.dtype == torch.float32 and t.is_contiguous()
+        cache = None
+        if self.phi_k_cache is not None:
+            assert self.phi_k_cache.dtype == torch.float32 and self.phi_k_cache.is_contiguous()
+            cache = self.phi_k_cache.data_ptr()
         return _PhiDesc(self.w_q.data_ptr(), self.b_q.data_ptr(), self.w_k.data_ptr(), self.b_k.data_ptr(),
-                        float(self.gamma_q), float(self.gamma_k))
+                        float(self.gamma_q), float(self.gamma_k), cache)
 
 
 def _topk_host(topk) -> np.ndarray:

@@ -126,6 +126,7 @@ void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, W
   if (L->max_slices < 1) L->max_slices = 1;
   L->partial_stride = 4 + 2 * kv->head_dim;
   L->partials = o;      o = align_up(o + sizeof(float) * (size_t)sh.rows * L->max_slices * L->partial_stride, 256);
+  L->zbuf = o;          o = align_up(o + sizeof(float) * (size_t)sh.rows * (topk_max > 0 ? topk_max : 1), 256);
   L->total = o;
 }
 
@@ -261,6 +262,8 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
       return fail(TKPHI_ERR_INVALID_ARG, "w_q, w_k, S and u must be 16-byte aligned");
     if (!std::isfinite(phi->gamma_q) || !std::isfinite(phi->gamma_k))
       return fail(TKPHI_ERR_INVALID_ARG, "gamma must be finite");
+    if (phi->phi_k_cache && !aligned16(phi->phi_k_cache))
+      return fail(TKPHI_ERR_INVALID_ARG, "phi_k_cache must be 16-byte aligned");
   }
   WsLayout L{};
   decode_layout(kv, sh, topk_max, &L);
@@ -281,7 +284,12 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   if (with_phi) {
     p.w_q = phi->w_q; p.b_q = phi->b_q; p.w_k = phi->w_k; p.b_k = phi->b_k;
     p.gamma_q = phi->gamma_q; p.gamma_k = phi->gamma_k; p.S = S; p.u = u;
+    if (phi->phi_k_cache && !(flags & TKPHI_FLAG_NOSUB)) {
+      p.phi_cache = phi->phi_k_cache;
+      p.zbuf = reinterpret_cast<float*>(w + L.zbuf);
+    }
   }
+  p.total_tokens = sh.total_tokens;
   p.idx_out = idx_out; p.y_out = y_out; p.dbg_out = dbg_out; p.flags = flags; p.with_phi = with_phi ? 1 : 0;
   p.status = reinterpret_cast<int*>(w + L.status);
   p.row_counter = reinterpret_cast<unsigned*>(w + L.row_counter);
@@ -318,6 +326,11 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
     e = launch_select(p, sh.score_tiles > 0 ? sh.max_mid : 0, n_sm_cached(), cs);
   }
   if (e != cudaSuccess) return cuda_fail(e, "select launch");
+  if (p.zbuf) {
+    ScopedSpan sp(cs, TKPHI_KERNEL_CACHED_Z);
+    e = launch_cached_z(p, cs);
+    if (e != cudaSuccess) return cuda_fail(e, "cached-feature launch");
+  }
   {
     ScopedSpan sp(cs, TKPHI_KERNEL_EXACT_RESIDUAL);
     // slice pairs of the whole call (two 128-token slices of a support list per CTA)
@@ -419,11 +432,14 @@ tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc
   p.k = static_cast<const __nv_bfloat16*>(kv->k); p.v = static_cast<const __nv_bfloat16*>(kv->v);
   p.stride_head = kv->kv_stride_head; p.stride_token = kv->kv_stride_token;
   p.w_k = phi->w_k; p.b_k = phi->b_k; p.gamma_k = phi->gamma_k;
+  p.phi_cache = phi->phi_k_cache; p.total_tokens = sh.total_tokens;
   p.S = S; p.u = u;
   p.status = reinterpret_cast<int*>(w + L.status);
   p.partials = reinterpret_cast<float*>(w + L.b_partials);
   p.chunks_per_unit = L.chunks_per_unit;
   if (!aligned16(phi->w_k)) return fail(TKPHI_ERR_INVALID_ARG, "w_k must be 16-byte aligned");
+  if (phi->phi_k_cache && !aligned16(phi->phi_k_cache))
+    return fail(TKPHI_ERR_INVALID_ARG, "phi_k_cache must be 16-byte aligned");
   CUtensorMap tk, tv;
   st = make_tensor_map(kv, kv->k, 128, sh.total_tokens, &tk);
   if (st != TKPHI_OK) return st;

@@ -15,6 +15,8 @@
 //            straight from tensor memory; B operand: the value tile as TMA lands it
 //            (tokens along K, dims contiguous).  S^T accumulates in tensor memory over
 //            all tiles of the CTA.
+// With a feature cache (Sec. 4.2 notes that a cached implementation avoids the decode-side
+// recompute) the feature warps also write every phi_k row they produce to global memory.
 // Warp roles: 0 TMA producer, 1 MMA issuer, 2..9 feature warps, 10..13 key norms.
 // GEMM 1 of tile i+1 is issued before GEMM 2 of tile i, so the tensor pipe works while
 // the feature warps are busy.  Each CTA owns a contiguous range of tiles of one
@@ -242,6 +244,9 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     const int j = quad * 32 + lane;                // feature
     const float bj = j < R ? p.b_k[(size_t)kvh * R + j] * kLog2e : 0.f;
     float u_acc = 0.f;                             // sum of feature j over this thread's tokens
+    // optional cached features: row of mid token 0 of this head, column j
+    float* cache_j = (p.phi_cache && j < R)
+                         ? p.phi_cache + ((size_t)kvh * p.total_tokens + (size_t)row0) * R + j : nullptr;
     bool ok = true;
     for (int it = 0; it < n_my && ok; ++it) {
       const int buf = it & 1;
@@ -268,6 +273,12 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
               __floats2bfloat162_rn(f0 - __bfloat162float(hp.x), f1 - __bfloat162float(hp.y));
           hi[e] = *reinterpret_cast<const uint32_t*>(&hp);
           lo[e] = *reinterpret_cast<const uint32_t*>(&lp);
+          if (cache_j) {
+            // one token per store: the 32 lanes of the warp write 32 consecutive features
+            const int tok = (t0 + it) * kBT + h * 64 + c * 32 + 2 * e;
+            if (tok < n_mid) __stcs(cache_j + (size_t)tok * R, f0);
+            if (tok + 1 < n_mid) __stcs(cache_j + (size_t)(tok + 1) * R, f1);
+          }
         }
         // hi goes over columns of this thread's own region that it has already read
         tmem_st_x16(tmem_addr(tmem_base, quad * 32, kColD1 + buf * 128 + h * 64 + c * 16), hi);

@@ -34,6 +34,10 @@ struct Problem {
   // feature maps
   const float* w_q; const float* b_q; const float* w_k; const float* b_k;
   float gamma_q, gamma_k;
+  // cached key features (optional): phi_k rows [n_kv_heads][total_tokens][n_feat], and where the
+  // decode step keeps z_i = <phi_q, phi_k(k_i)> / exp(m_q) of the retrieved tokens: [rows][topk_max]
+  const float* phi_cache; long long total_tokens;
+  float* zbuf;                     // null: the features of the retrieved keys are recomputed
   // summaries
   const float* S; const float* u;
   // row gather of the exact support through 2-D tensor maps over the k and v caches:
@@ -64,6 +68,8 @@ struct BuildProblem {
   const __nv_bfloat16* v;
   long long stride_head, stride_token;
   const float* w_k; const float* b_k; float gamma_k;
+  float* phi_cache;                // optional: phi_k rows of the mid-region tokens are also written here
+  long long total_tokens;
   float* S; float* u;
   int* status;
   float* partials;                 // [units][chunks_per_unit][d*r + r]
@@ -73,7 +79,7 @@ struct BuildProblem {
 // Host-side byte offsets of the workspace pieces.
 struct WsLayout {
   size_t status, row_counter, zero_end;
-  size_t scores, wk_img, idx, aq, partials, total;
+  size_t scores, wk_img, idx, aq, partials, zbuf, total;
   int max_slices, partial_stride;
   // build
   size_t b_partials; int chunks_per_unit;
@@ -182,6 +188,7 @@ cudaError_t launch_score(const Problem& p, const CUtensorMap& tmap_k, int n_sm, 
 cudaError_t launch_select(const Problem& p, int max_mid, int n_sm, cudaStream_t stream);
 cudaError_t launch_exact_residual(const Problem& p, const CUtensorMap& gk, const CUtensorMap& gv, long long n_pairs, int n_sm,
                                   cudaStream_t stream);
+cudaError_t launch_cached_z(const Problem& p, cudaStream_t stream);
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, cudaStream_t stream);
 
 }  // namespace tkphi

@@ -26,6 +26,10 @@
 // cross-thread reduction.  Each CTA writes partial sums; the last CTA of a head (one atomic
 // ticket, no spinning) combines them in slice order, so results are run-to-run
 // identical.
+//
+// With cached key features (Sec. 4.2 mentions a cached implementation; cached_features.cu) the z_i of
+// the retrieved tokens come from a buffer instead: no key rows of retrieved tokens, no W_k tiles, no
+// tensor-core work; everything else is the same.
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -51,6 +55,97 @@ struct ExSmem {
   //        red[groups][4*D], misc[32]
   static constexpr size_t total = small + 32 + 4 * (4 * kExThreads + D + 2 * R + kExGroups * 4 * D + 32);
 };
+
+// ------------------------------------------------------------------ per-slice arithmetic shared by both kernels
+// Thread = token `gt` of a 128-token slice whose k rows sit in the 128B-swizzled tile `kt`:
+// returns q . k_t / sqrt(d) (*dot_scaled) and |k_t|^2 (*kn).
+template <int D>
+__device__ __forceinline__ void token_dot_and_norm(const unsigned char* kt, int gt, const float* qf, float scale,
+                                                   float* dot_scaled, float* kn_out) {
+  using L = ExSmem<D, 64>;                                  // (tile geometry does not depend on R)
+  float dot = 0.f, kn = 0.f;
+#pragma unroll
+  for (int c = 0; c < D / 8; ++c) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(kt + (c >> 3) * L::KV_BOX + swz128(gt, c & 7));
+    const unsigned w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float x0 = bf16_lo(w[e]), x1 = bf16_hi(w[e]);
+      dot = fmaf(x0, qf[c * 8 + 2 * e], dot);
+      dot = fmaf(x1, qf[c * 8 + 2 * e + 1], dot);
+      kn = fmaf(x0, x0, kn);
+      kn = fmaf(x1, x1, kn);
+    }
+  }
+  *dot_scaled = dot * scale;
+  *kn_out = kn;
+}
+
+// z_t = <phi_q, phi_k(k_t)> / exp(m_q) from this token's row of the feature-recompute accumulator
+// (columns [0, R): W_hi k_t, [R, 2R): W_lo k_t, both scaled by log2 e; lane of tensor memory = token):
+// z = 2^(-gamma log2e |k|^2) * sum_j 2^(hi_j + lo_j + c_j), c_j = log2 w_j + b_k[j] log2 e; four partial
+// sums in a fixed order.  Called by whole warps (gwarp = warp index inside the slice's group).
+template <int R>
+__device__ __forceinline__ float z_from_accumulator(uint32_t tmem_d, int gwarp, const float* cj, float gamma_k, float kn) {
+  float zp[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int c4 = 0; c4 < R / 32; ++c4) {
+    float v[32], vl[32];
+    tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, c4 * 32), v);
+    tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, R + c4 * 32), vl);
+    tc_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) zp[j & 3] += ex2_approx((v[j] + vl[j]) + cj[c4 * 32 + j]);
+  }
+  return ((zp[0] + zp[1]) + (zp[2] + zp[3])) * ex2_approx(-gamma_k * kLog2e * kn);
+}
+
+// Value pass of one slice (thread gt of its group): nu[dv] = sum_t w_t v_t[dv], zv[dv] = sum_t z_t v_t[dv]
+// over the thread's token group, even / odd tokens added in a fixed order, into red[tg][2 D].
+template <int D>
+__device__ __forceinline__ void slice_value_pass(const unsigned char* vt, const float* wgt, const float* zt, int gt,
+                                                 float* red) {
+  using L = ExSmem<D, 64>;
+  constexpr int NGV = kSlice / D;            // token groups for the value pass (1 or 2)
+  constexpr int TPV = kSlice / NGV;
+  const int dv = gt % D, tg = gt / D;
+  const unsigned char* vcol = vt + (dv >> 6) * L::KV_BOX + (dv & 7) * 2;
+  const uint32_t ch = (dv & 63) >> 3;
+  float nu0 = 0.f, nu1 = 0.f, zv0 = 0.f, zv1 = 0.f;
+#pragma unroll 4
+  for (int t = tg * TPV; t < (tg + 1) * TPV; t += 2) {
+    const unsigned short r0 = *reinterpret_cast<const unsigned short*>(vcol + swz128(t, ch));
+    const unsigned short r1 = *reinterpret_cast<const unsigned short*>(vcol + swz128(t + 1, ch));
+    const float x0 = __uint_as_float((unsigned)r0 << 16), x1 = __uint_as_float((unsigned)r1 << 16);
+    nu0 = fmaf(wgt[t], x0, nu0);
+    zv0 = fmaf(zt[t], x0, zv0);
+    nu1 = fmaf(wgt[t + 1], x1, nu1);
+    zv1 = fmaf(zt[t + 1], x1, zv1);
+  }
+  red[tg * 2 * D + dv] = nu0 + nu1;
+  red[tg * 2 * D + D + dv] = zv0 + zv1;
+}
+
+// Writes a slice's partial sums: part[0..3] = m_slice, Z = sum w_t, zs = sum z_t, 0; part[4..] = nu, zv.
+// Called by the 128 threads of the slice's group after slice_value_pass and a barrier.
+template <int D>
+__device__ __forceinline__ void slice_write_partials(float* part, const float* red, const float* wgt, const float* zt,
+                                                     int gt, int gwarp, int lane, float m_slice) {
+  constexpr int NGV = kSlice / D;
+  for (int i = gt; i < 2 * D; i += kSlice) {
+    float x = red[i];
+    if (NGV == 2) x += red[2 * D + i];       // second token group, fixed order
+    part[4 + i] = x;
+  }
+  if (gwarp == 0) {
+    float Z = 0.f, zs = 0.f;
+#pragma unroll
+    for (int i = 0; i < kSlice / 32; ++i) { Z += wgt[lane + 32 * i]; zs += zt[lane + 32 * i]; }
+    Z = warp_sum(Z);
+    zs = warp_sum(zs);
+    if (lane == 0) { part[0] = m_slice; part[1] = Z; part[2] = zs; part[3] = 0.f; }
+  }
+}
 
 // The last CTA of a head combines the slice partials in slice order, by a fixed assignment
 // of slices to lanes and of output columns to threads, so the result does not depend on
@@ -211,8 +306,8 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   if (slice0 >= n_slices) return;
   const int n_ctas = (n_slices + kExGroups - 1) / kExGroups;
   const bool live = slice < n_slices;            // the last CTA of a head may hold one empty group
-  const bool do_phi = p.with_phi && !(p.flags & 1u);
-  // does a slice hold retrieved tokens (positions nA1 .. nA1+K-1 of the support list)?
+  const bool do_phi = p.with_phi && !(p.flags & 1u) && !p.zbuf;   // recompute the retrieved keys' features here
+  // does a slice hold retrieved tokens (positions nA1 .. nA1+K-1 of the support list) whose features are recomputed?
   auto slice_has_ret = [&](int s) { return do_phi && s < n_slices && s * kSlice < nA1 + K && (s + 1) * kSlice > nA1; };
   const bool has_ret = slice_has_ret(slice);
   bool any_ret = false;
@@ -234,6 +329,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   pdl_wait();                                  // the index lists, features and score rows of the predecessors
   if (any_ret && warp == 0) tmem_alloc(s_tmem, kExGroups * 2 * R);   // after the wait: never hold columns a predecessor needs
   // ---- 1. token list of this slice
+  float z_cached = 0.f;                        // cached features: z of this thread's token
   {
     const int pi = slice * kSlice + gt;
     int t = -1, ret = 0;
@@ -244,6 +340,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
     }
     tok[gt] = t;
     isret[gt] = ret;
+    if (ret && p.zbuf) z_cached = __ldcg(p.zbuf + (size_t)row * p.topk_max + (pi - nA1));   // used in step 5
   }
   for (int c = tid; c < D; c += kExThreads) qf[c] = __bfloat162float(p.q[(size_t)row * D + c]);
   if (do_phi) {
@@ -310,21 +407,9 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   const int ti = tok[gt];
   float s_val = -INFINITY, kn = 0.f;
   if (ti >= 0) {
-    float dot = 0.f;
-#pragma unroll
-    for (int c = 0; c < CPR; ++c) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(kt + (c >> 3) * L::KV_BOX + swz128(gt, c & 7));
-      const unsigned w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float x0 = bf16_lo(w[e]), x1 = bf16_hi(w[e]);
-        dot = fmaf(x0, qf[c * 8 + 2 * e], dot);
-        dot = fmaf(x1, qf[c * 8 + 2 * e + 1], dot);
-        kn = fmaf(x0, x0, kn);
-        kn = fmaf(x1, x1, kn);
-      }
-    }
-    s_val = isret[gt] ? srow[ti - p.n_sink] : dot * p.scale;
+    float dot;
+    token_dot_and_norm<D>(kt, gt, qf, p.scale, &dot, &kn);
+    s_val = isret[gt] ? srow[ti - p.n_sink] : dot;
   }
   {
     const float m = warp_max(s_val);
@@ -348,64 +433,19 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   }
   if (has_ret && ok) {
     tc_fence_after_sync();
-    const uint32_t tmem_d = *s_tmem + grp * 2 * R;
-    // z = 2^(-gamma log2e |k|^2) * sum_j 2^(hi_j + lo_j + c_j): four partial sums in a fixed order
-    float zp[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int c4 = 0; c4 < R / 32; ++c4) {
-      float v[32], vl[32];
-      tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, c4 * 32), v);
-      tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, R + c4 * 32), vl);
-      tc_wait_ld();
-#pragma unroll
-      for (int j = 0; j < 32; ++j) zp[j & 3] += ex2_approx((v[j] + vl[j]) + cj[c4 * 32 + j]);
-    }
-    z_t = ((zp[0] + zp[1]) + (zp[2] + zp[3])) * ex2_approx(-p.gamma_k * kLog2e * kn);
+    z_t = z_from_accumulator<R>(*s_tmem + grp * 2 * R, gwarp, cj, p.gamma_k, kn);
     if (!isret[gt]) z_t = 0.f;
   }
+  if (p.zbuf) z_t = z_cached;                  // (zero for anchors)
   zt[gt] = z_t;
   __syncthreads();
 
   // ---- 6. slice partials: nu = sum w_t v_t, zv = sum z_t v_t, Z = sum w_t, zs = sum z_t
-  {
-    constexpr int NGV = kSlice / D;          // token groups for the value pass (1 or 2)
-    constexpr int TPV = kSlice / NGV;
-    const int dv = gt % D, tg = gt / D;
-    const unsigned char* vcol = vt + (dv >> 6) * L::KV_BOX + (dv & 7) * 2;
-    const uint32_t ch = (dv & 63) >> 3;
-    float nu0 = 0.f, nu1 = 0.f, zv0 = 0.f, zv1 = 0.f;      // even / odd tokens, added in a fixed order
-#pragma unroll 4
-    for (int t = tg * TPV; t < (tg + 1) * TPV; t += 2) {
-      const unsigned short r0 = *reinterpret_cast<const unsigned short*>(vcol + swz128(t, ch));
-      const unsigned short r1 = *reinterpret_cast<const unsigned short*>(vcol + swz128(t + 1, ch));
-      const float x0 = __uint_as_float((unsigned)r0 << 16), x1 = __uint_as_float((unsigned)r1 << 16);
-      nu0 = fmaf(wgt[t], x0, nu0);
-      zv0 = fmaf(zt[t], x0, zv0);
-      nu1 = fmaf(wgt[t + 1], x1, nu1);
-      zv1 = fmaf(zt[t + 1], x1, zv1);
-    }
-    const float nu = nu0 + nu1, zv = zv0 + zv1;
-    red[tg * 2 * D + dv] = nu;
-    red[tg * 2 * D + D + dv] = zv;
-  }
+  slice_value_pass<D>(vt, wgt, zt, gt, red);
   __syncthreads();
-  float* part = p.partials + ((size_t)row * p.max_slices + slice) * p.partial_stride;
-  if (live) {
-    for (int i = gt; i < 2 * D; i += kSlice) {
-      constexpr int NGV = kSlice / D;
-      float x = red[i];
-      if (NGV == 2) x += red[2 * D + i];     // second token group, fixed order
-      part[4 + i] = x;
-    }
-    if (gwarp == 0) {
-      float Z = 0.f, zs = 0.f;
-#pragma unroll
-      for (int i = 0; i < kSlice / 32; ++i) { Z += wgt[lane + 32 * i]; zs += zt[lane + 32 * i]; }
-      Z = warp_sum(Z);
-      zs = warp_sum(zs);
-      if (lane == 0) { part[0] = m_slice; part[1] = Z; part[2] = zs; part[3] = 0.f; }
-    }
-  }
+  if (live)
+    slice_write_partials<D>(p.partials + ((size_t)row * p.max_slices + slice) * p.partial_stride, red, wgt, zt, gt, gwarp,
+                            lane, m_slice);
 
   // ---- tensor memory is no longer needed
   tc_fence_before_sync();
@@ -454,9 +494,9 @@ struct ExStreamSmem {
   static constexpr size_t vt = w + B::w_bytes;
   static constexpr size_t small = vt + kExGroups * B::kv_tile;
   // small: bars[8], tok[2][T] int, isret[2][T] int, wgt[T], zt[T], qf[2][D], cj[2][R], red[groups][4*D],
-  //        misc[32], pre[kMaxBatch + 2] int
+  //        misc[32], pre[kMaxBatch + 2] int, zc[2][T]
   static constexpr size_t total =
-      small + 64 + 4 * (6 * kExThreads + 2 * D + 2 * R + kExGroups * 4 * D + 32 + kMaxBatch + 2);
+      small + 64 + 4 * (8 * kExThreads + 2 * D + 2 * R + kExGroups * 4 * D + 32 + kMaxBatch + 2);
 };
 
 constexpr int kExStreamThreads = kExThreads + 64;   // compute warps 0..7, producer warps 8 (k rows) and 9 (v rows)
@@ -493,9 +533,10 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 28);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 29);
   int* pre = reinterpret_cast<int*>(misc + 32);                     // [batch + 1] items before sequence b
+  float* zc_all = reinterpret_cast<float*>(pre + kMaxBatch + 2);    // [2 buffers][T] cached z of the tokens
 
   pdl_launch_next();
-  const bool do_phi = p.with_phi && !(p.flags & 1u);
+  const bool do_phi = p.with_phi && !(p.flags & 1u) && !p.zbuf;     // recompute the retrieved keys' features here
   const int batch = p.batch, Hq = p.n_q_heads;
 
   // ---- items per sequence -> prefix (reads only the call's inputs)
@@ -579,15 +620,19 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
   // token list, queries and query-side feature terms of an item: loaded into registers first
   // (stage_load) and written to buffer `buf` later (stage_store), so that the loads of the next
   // item are in flight while the current one is computed.  D, R <= kExThreads: one value each.
-  struct Staged { int t, ret; float qv, cv; };
+  struct Staged { int t, ret; float qv, cv, zc; };
   auto stage_load = [&](const ExItem& it) {
     Staged sg;
     const int sl = it.slice0 + grp;
     const int pi = sl * kSlice + gt;
-    sg.t = -1; sg.ret = 0;
+    sg.t = -1; sg.ret = 0; sg.zc = 0.f;
     if (sl < it.n_slices && pi < it.nE) {
       if (pi < it.nA1) sg.t = pi;
-      else if (pi < it.nA1 + it.K) { sg.t = __ldcg(p.idx + (size_t)it.row * p.topk_max + (pi - it.nA1)); sg.ret = 1; }
+      else if (pi < it.nA1 + it.K) {
+        sg.t = __ldcg(p.idx + (size_t)it.row * p.topk_max + (pi - it.nA1));
+        sg.ret = 1;
+        if (p.zbuf) sg.zc = __ldcg(p.zbuf + (size_t)it.row * p.topk_max + (pi - it.nA1));
+      }
       else sg.t = it.tail_start + (pi - it.nA1 - it.K);
     }
     sg.qv = tid < D ? __bfloat162float(p.q[(size_t)it.row * D + tid]) : 0.f;
@@ -599,6 +644,7 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
   auto stage_store = [&](const Staged& sg, int buf) {
     tok_all[buf * kExThreads + tid] = sg.t;
     isret_all[buf * kExThreads + tid] = sg.ret;
+    zc_all[buf * kExThreads + tid] = sg.zc;
     if (tid < D) qf_all[buf * D + tid] = sg.qv;
     if (tid < R) cj_all[buf * R + tid] = sg.cv;
   };
@@ -723,7 +769,7 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
     // ---- next item: token list and query terms into the other buffer
     ExItem nxt = cur;
     const bool has_next = i + 1 < i1;
-    Staged sg_next{-1, 0, 0.f, 0.f};
+    Staged sg_next{-1, 0, 0.f, 0.f, 0.f};
     if (has_next) { nxt = item_of(i + 1, &cur); sg_next = stage_load(nxt); }
 
     // ---- k tiles of this item have landed (the v tiles may still be in flight)
@@ -757,21 +803,9 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
     const int ti = tok[gt];
     float s_val = -INFINITY, kn = 0.f;
     if (ti >= 0) {
-      float dot = 0.f;
-#pragma unroll
-      for (int c = 0; c < CPR; ++c) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(kt + (c >> 3) * LB::KV_BOX + swz128(gt, c & 7));
-        const unsigned wv[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float x0 = bf16_lo(wv[e]), x1 = bf16_hi(wv[e]);
-          dot = fmaf(x0, qf[c * 8 + 2 * e], dot);
-          dot = fmaf(x1, qf[c * 8 + 2 * e + 1], dot);
-          kn = fmaf(x0, x0, kn);
-          kn = fmaf(x1, x1, kn);
-        }
-      }
-      s_val = isret[gt] ? srow[ti - p.n_sink] : dot * p.scale;
+      float dot;
+      token_dot_and_norm<D>(kt, gt, qf, p.scale, &dot, &kn);
+      s_val = isret[gt] ? srow[ti - p.n_sink] : dot;
     }
     {
       const float m = warp_max(s_val);
@@ -794,64 +828,21 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
     float z_t = 0.f;
     if (has_ret && ok) {
       tc_fence_after_sync();
-      const uint32_t tmem_d = *s_tmem + grp * 2 * R;
-      float zp[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int c4 = 0; c4 < R / 32; ++c4) {
-        float v[32], vl[32];
-        tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, c4 * 32), v);
-        tmem_ld_x32(tmem_addr(tmem_d, gwarp * 32, R + c4 * 32), vl);
-        tc_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) zp[j & 3] += ex2_approx((v[j] + vl[j]) + cj[c4 * 32 + j]);
-      }
-      z_t = ((zp[0] + zp[1]) + (zp[2] + zp[3])) * ex2_approx(-p.gamma_k * kLog2e * kn);
+      z_t = z_from_accumulator<R>(*s_tmem + grp * 2 * R, gwarp, cj, p.gamma_k, kn);
       if (!isret[gt]) z_t = 0.f;
     }
+    if (p.zbuf) z_t = zc_all[buf * kExThreads + tid];
     zt[gt] = z_t;
     tc_fence_before_sync();                    // the accumulator reads precede the next item's MMAs
     ex_sync<1>();
 
     // ---- slice partials
-    {
-      constexpr int NGV = kSlice / D;
-      constexpr int TPV = kSlice / NGV;
-      const int dv = gt % D, tg = gt / D;
-      const unsigned char* vcol = vt + (dv >> 6) * LB::KV_BOX + (dv & 7) * 2;
-      const uint32_t ch = (dv & 63) >> 3;
-      float nu0 = 0.f, nu1 = 0.f, zv0 = 0.f, zv1 = 0.f;
-#pragma unroll 4
-      for (int t = tg * TPV; t < (tg + 1) * TPV; t += 2) {
-        const unsigned short r0 = *reinterpret_cast<const unsigned short*>(vcol + swz128(t, ch));
-        const unsigned short r1 = *reinterpret_cast<const unsigned short*>(vcol + swz128(t + 1, ch));
-        const float x0 = __uint_as_float((unsigned)r0 << 16), x1 = __uint_as_float((unsigned)r1 << 16);
-        nu0 = fmaf(wgt[t], x0, nu0);
-        zv0 = fmaf(zt[t], x0, zv0);
-        nu1 = fmaf(wgt[t + 1], x1, nu1);
-        zv1 = fmaf(zt[t + 1], x1, zv1);
-      }
-      red[tg * 2 * D + dv] = nu0 + nu1;
-      red[tg * 2 * D + D + dv] = zv0 + zv1;
-    }
+    slice_value_pass<D>(vt, wgt, zt, gt, red);
     ok = ex_sync_and<1>(ok);                   // the v tiles are free for the next item
     if (tid == 0) mbar_arrive(&bars[6]);
-    if (live) {
-      float* part = p.partials + ((size_t)cur.row * p.max_slices + slice) * p.partial_stride;
-      for (int c = gt; c < 2 * D; c += kSlice) {
-        constexpr int NGV = kSlice / D;
-        float x = red[c];
-        if (NGV == 2) x += red[2 * D + c];
-        part[4 + c] = x;
-      }
-      if (gwarp == 0) {
-        float Z = 0.f, zs = 0.f;
-#pragma unroll
-        for (int c = 0; c < kSlice / 32; ++c) { Z += wgt[lane + 32 * c]; zs += zt[lane + 32 * c]; }
-        Z = warp_sum(Z);
-        zs = warp_sum(zs);
-        if (lane == 0) { part[0] = m_slice; part[1] = Z; part[2] = zs; part[3] = 0.f; }
-      }
-    }
+    if (live)
+      slice_write_partials<D>(p.partials + ((size_t)cur.row * p.max_slices + slice) * p.partial_stride, red, wgt, zt, gt,
+                              gwarp, lane, m_slice);
     if (!ok) break;                            // a wait gave up (the same for every thread)
 
     // ---- ticket: the last CTA of this head merges

@@ -103,7 +103,7 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
       __threadfence_block();
       __syncthreads();
       phi_q_stage2<kSelThreads>(p, task);
-    } else if (task < n_rows + p.n_kv_heads && !(p.flags & 1u)) {
+    } else if (task < n_rows + p.n_kv_heads && !(p.flags & 1u) && !p.zbuf) {   // (cached features need no W_k tiles)
       wk_split_job<kSelThreads>(p, task - n_rows);
     }
     return;

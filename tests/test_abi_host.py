@@ -84,14 +84,15 @@ def test_invalid_arguments_are_rejected_before_any_launch(lib):
 def test_decode_step_and_build_validation(lib):
     d, cu = _desc([0, 400])
     topk = np.array([3], np.int32)
-    ph = B._PhiDesc(0x100, 0x200, 0x300, 0x400, 0.5, 0.5)
+    ph = B._PhiDesc(0x100, 0x200, 0x300, 0x400, 0.5, 0.5, None)
     args = lambda **kw: (C.byref(d), C.byref(kw.get("ph", ph)), 0x4000, topk.ctypes.data, 0x6000, 3,
                          kw.get("S", 0x7000), 0x8000, None, 0x5000, None, kw.get("flags", 0),
                          kw.get("ws", 0x10000), kw.get("wsb", 1 << 40), None)
     assert lib.tkphi_decode_step(*args(S=0)) == -1
     assert lib.tkphi_decode_step(*args(flags=8)) == -1
-    assert lib.tkphi_decode_step(*args(ph=B._PhiDesc(0, 0x200, 0x300, 0x400, 0.5, 0.5))) == -1
-    assert lib.tkphi_decode_step(*args(ph=B._PhiDesc(0x100, 0x200, 0x300, 0x400, float("nan"), 0.5))) == -1
+    assert lib.tkphi_decode_step(*args(ph=B._PhiDesc(0, 0x200, 0x300, 0x400, 0.5, 0.5, None))) == -1
+    assert lib.tkphi_decode_step(*args(ph=B._PhiDesc(0x100, 0x200, 0x300, 0x400, float("nan"), 0.5, None))) == -1
+    assert lib.tkphi_decode_step(*args(ph=B._PhiDesc(0x100, 0x200, 0x300, 0x400, 0.5, 0.5, 0x9008))) == -1   # misaligned cache
     assert lib.tkphi_decode_step(*args(wsb=1000)) == -3
     assert lib.tkphi_build_summaries(C.byref(d), C.byref(ph), 0, 0x8000, 0x10000, 1 << 40, None) == -1
     assert lib.tkphi_build_summaries(C.byref(d), None, 0x7000, 0x8000, 0x10000, 1 << 40, None) == -1

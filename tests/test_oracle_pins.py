@@ -296,6 +296,33 @@ def test_rel_l1_hand_computed_cases(golden):
     assert O.rel_l1([0.25, 0.5], [0.25, 0.5]) == 0.0
 
 
+def test_cached_features_equal_recomputed_features():
+    # Sec. 4.2: a cache of phi_k rows written at build time gives the same Top-K+phi output as recomputing
+    # the retrieved keys' features; summaries built from the same cached rows cancel exactly at K = |M|
+    p = _rand_problem(21)
+    Phi = O.phi(p["K"], p["Wk"], p["bk"], 0.5)
+    S, u = O.build_summaries(p["K"], p["V"], p["Wk"], p["bk"], 0.5, 2, 3)
+    ref = O.topkphi_attention(p["q"], p["K"], p["V"], 2, 3, 9, p["Wq"], p["bq"], 0.5, p["Wk"], p["bk"], 0.5, S=S, u=u)
+    got = O.topkphi_attention_cached(p["q"], p["K"], p["V"], 2, 3, 9, p["Wq"], p["bq"], 0.5, Phi, S, u)
+    np.testing.assert_allclose(got.y, ref.y, rtol=1e-14, atol=0)
+    assert got.retrieved.tolist() == ref.retrieved.tolist() and abs(got.log_Zhat_R - ref.log_Zhat_R) < 1e-13
+    # rows outside the retrieved set are never read: garbage there changes nothing
+    junk = Phi.copy()
+    mask = np.ones(len(Phi), bool); mask[ref.retrieved] = False
+    junk[mask] = 1e30
+    np.testing.assert_array_equal(
+        O.topkphi_attention_cached(p["q"], p["K"], p["V"], 2, 3, 9, p["Wq"], p["bq"], 0.5, junk, S, u).y, got.y)
+    # a cache whose rows are off by one token is a different (wrong) estimator
+    shifted = np.roll(Phi, 1, axis=0)
+    bad = O.topkphi_attention_cached(p["q"], p["K"], p["V"], 2, 3, 9, p["Wq"], p["bq"], 0.5, shifted, S, u)
+    assert np.abs(bad.y - ref.y).max() > 1e-6
+    # K = |M| with summaries built from the cached rows: the residual cancels and y is full attention
+    S2, u2 = O.build_summaries_from_features(p["V"], Phi, 2, 3)
+    full = O.topkphi_attention_cached(p["q"], p["K"], p["V"], 2, 3, 35, p["Wq"], p["bq"], 0.5, Phi, S2, u2)
+    np.testing.assert_allclose(full.y, O.full_attention(p["q"], p["K"], p["V"]), rtol=1e-10)
+    assert np.abs(full.S_R).max() <= 1e-12 * np.abs(S2).max()
+
+
 def test_reassociated_form_equals_literal():
     p = _rand_problem(15)
     res = _run(p, 7)
