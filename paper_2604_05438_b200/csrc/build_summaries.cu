@@ -60,7 +60,7 @@ __device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[
       : "memory");
 }
 
-template <int D>
+template <int D, bool CACHE>
 __global__ void __launch_bounds__(kBuildThreads, 1)
 build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
              const BuildProblem p) {
@@ -245,8 +245,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     const float bj = j < R ? p.b_k[(size_t)kvh * R + j] * kLog2e : 0.f;
     float u_acc = 0.f;                             // sum of feature j over this thread's tokens
     // optional cached features: row of mid token 0 of this head, column j
-    float* cache_j = (p.phi_cache && j < R)
-                         ? p.phi_cache + ((size_t)kvh * p.total_tokens + (size_t)row0) * R + j : nullptr;
+    float* cache_j = (CACHE && j < R) ? p.phi_cache + ((size_t)kvh * p.total_tokens + (size_t)row0) * R + j : nullptr;
     bool ok = true;
     for (int it = 0; it < n_my && ok; ++it) {
       const int buf = it & 1;
@@ -273,7 +272,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
               __floats2bfloat162_rn(f0 - __bfloat162float(hp.x), f1 - __bfloat162float(hp.y));
           hi[e] = *reinterpret_cast<const uint32_t*>(&hp);
           lo[e] = *reinterpret_cast<const uint32_t*>(&lp);
-          if (cache_j) {
+          if (CACHE && cache_j) {
             // one token per store: the 32 lanes of the warp write 32 consecutive features
             const int tok = (t0 + it) * kBT + h * 64 + c * 32 + 2 * e;
             if (tok < n_mid) __stcs(cache_j + (size_t)tok * R, f0);
@@ -382,15 +381,15 @@ __global__ void __launch_bounds__(kRedThreads) build_reduce_kernel(const BuildPr
   }
 }
 
-template <int D>
+template <int D, bool CACHE>
 static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, const CUtensorMap& tv,
                                   cudaStream_t st) {
   static PerDeviceFlag configured;
   const size_t smem = BuildCfg<D>::total;
-  cudaError_t e = set_max_dynamic_smem(configured, reinterpret_cast<const void*>(build_kernel<D>), smem);
+  cudaError_t e = set_max_dynamic_smem(configured, reinterpret_cast<const void*>(build_kernel<D, CACHE>), smem);
   if (e != cudaSuccess) return e;
   dim3 grid(p.chunks_per_unit, p.n_kv_heads, p.batch);
-  build_kernel<D><<<grid, kBuildThreads, smem, st>>>(tk, tv, p);
+  build_kernel<D, CACHE><<<grid, kBuildThreads, smem, st>>>(tk, tv, p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   // one output per thread: every thread's loads of all chunk partials are in flight at once
@@ -400,8 +399,8 @@ static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, 
 }
 
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tk, const CUtensorMap& tv, cudaStream_t st) {
-  if (p.head_dim == 64) return launch_build_t<64>(p, tk, tv, st);
-  if (p.head_dim == 128) return launch_build_t<128>(p, tk, tv, st);
+  if (p.head_dim == 64) return p.phi_cache ? launch_build_t<64, true>(p, tk, tv, st) : launch_build_t<64, false>(p, tk, tv, st);
+  if (p.head_dim == 128) return p.phi_cache ? launch_build_t<128, true>(p, tk, tv, st) : launch_build_t<128, false>(p, tk, tv, st);
   return cudaErrorInvalidValue;
 }
 
