@@ -145,6 +145,43 @@ def phi(x, W, b, gamma: float) -> np.ndarray:
     return np.exp(phi_log(x, W, b, gamma))
 
 
+# --------------------------------------------------------------------------
+# App. C.2: the head-wise one-block ReZero MLP feature map
+# --------------------------------------------------------------------------
+def gelu(x):
+    """GeLU(x) = x Phi(x), Phi the standard normal CDF (the erf form)."""
+    x = np.asarray(x, F64)
+    erf = np.vectorize(math.erf, otypes=[F64])
+    return 0.5 * x * (1.0 + erf(x / math.sqrt(2.0)))
+
+
+def phi_mlp_log(x, W_s, b_s, W_1, b_1, W_2, b_2, alpha, W_o, b_o) -> np.ndarray:
+    """log phi(x) of the one-block ReZero MLP feature map (App. C.2), in the paper's order:
+
+        g0 = W_s x + b_s;  Delta = W_2 GeLU(W_1 g0 + b_1) + b_2;  g1 = g0 + alpha Delta;
+        phi(x) = exp(W_o g1 + b_o).
+
+    Rows of x are vectors.  W_s: [d_emb, d_h], W_1, W_2: [d_emb, d_emb], W_o: [d_phi, d_emb].
+    """
+    x = np.atleast_2d(np.asarray(x, F64))
+    g0 = x @ np.asarray(W_s, F64).T + np.asarray(b_s, F64)
+    delta = gelu(g0 @ np.asarray(W_1, F64).T + np.asarray(b_1, F64)) @ np.asarray(W_2, F64).T + np.asarray(b_2, F64)
+    g1 = g0 + float(alpha) * delta
+    return g1 @ np.asarray(W_o, F64).T + np.asarray(b_o, F64)
+
+
+def phi_mlp(x, W_s, b_s, W_1, b_1, W_2, b_2, alpha, W_o, b_o) -> np.ndarray:
+    """phi(x) > 0 of the ReZero MLP feature map; a single vector in gives a single vector out."""
+    out = np.exp(phi_mlp_log(x, W_s, b_s, W_1, b_1, W_2, b_2, alpha, W_o, b_o))
+    return out[0] if np.asarray(x).ndim == 1 else out
+
+
+def phi_mlp_param_count(d_h: int, d_phi: int, d_emb: int = 512, n_scalars: int = 2) -> int:
+    """Parameters of one head's map: stem, two d_emb x d_emb layers, output layer, each with its
+    bias, plus the scalars (the paper's counts are met with two: alpha and one it does not name)."""
+    return (d_h * d_emb + d_emb) + 2 * (d_emb * d_emb + d_emb) + (d_emb * d_phi + d_phi) + n_scalars
+
+
 def build_summaries_from_features(V, Phi_k, n_sink: int, n_tail: int):
     """S_M = sum_{i in M} v_i phi_k(k_i)^T  (d_v x d_phi),  u_M = sum_{i in M} phi_k(k_i).
 

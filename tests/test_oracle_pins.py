@@ -323,6 +323,62 @@ def test_cached_features_equal_recomputed_features():
     assert np.abs(full.S_R).max() <= 1e-12 * np.abs(S2).max()
 
 
+def _mlp_params(seed, d=5, emb=7, r=4):
+    g = RNG(seed)
+    return dict(W_s=g.standard_normal((emb, d)) / math.sqrt(d), b_s=0.1 * g.standard_normal(emb),
+                W_1=g.standard_normal((emb, emb)) / math.sqrt(emb), b_1=0.1 * g.standard_normal(emb),
+                W_2=g.standard_normal((emb, emb)) / math.sqrt(emb), b_2=0.1 * g.standard_normal(emb),
+                alpha=0.37, W_o=g.standard_normal((r, emb)) / math.sqrt(emb), b_o=0.1 * g.standard_normal(r))
+
+
+def test_phi_mlp_parameter_counts_match_paper(golden):
+    # App. C.2 with hidden width 512; the table's four per-head counts and the two totals pin the layer shapes
+    assert O.phi_mlp_param_count(64, 32) == golden["phi_params_1b_dphi32"]
+    assert O.phi_mlp_param_count(64, 64) == golden["phi_params_1b_dphi64"]
+    assert O.phi_mlp_param_count(64, 128) == golden["phi_params_1b_dphi128"]
+    assert O.phi_mlp_param_count(128, 64) == golden["phi_params_3b_dphi64"]
+    assert round((512 + 128) * O.phi_mlp_param_count(64, 64) / 1e6, 1) == golden["phi_total_1b_dphi64_M"]
+    assert round((672 + 224) * O.phi_mlp_param_count(128, 64) / 1e6, 1) == golden["phi_total_3b_dphi64_M"]
+    # the arrays of a map add up to the count less the scalars the equations do not show
+    P = _mlp_params(0, d=64, emb=512, r=64)
+    n = sum(np.asarray(v).size for k, v in P.items() if k != "alpha")
+    assert n + 2 == O.phi_mlp_param_count(64, 64)
+
+
+def test_gelu_tabulated_values():
+    # x Phi(x) with the normal CDF at textbook points: Phi(1) = 0.8413447461, Phi(2) = 0.9772498681
+    np.testing.assert_allclose(O.gelu([0.0, 1.0, -1.0, 2.0, -2.0]),
+                               [0.0, 0.8413447461, -0.1586552539, 1.9544997361, -0.0455002639], atol=5e-10)
+    x = np.linspace(-4, 4, 33)
+    np.testing.assert_allclose(O.gelu(x) - O.gelu(-x), x, rtol=0, atol=1e-14)       # GeLU(x) - GeLU(-x) = x
+    assert abs(O.gelu(30.0) - 30.0) < 1e-12 and abs(O.gelu(-30.0)) < 1e-12
+
+
+def test_phi_mlp_reduces_to_affine_map_and_matches_scalar_loop():
+    P = _mlp_params(1)
+    g = RNG(2)
+    x = g.standard_normal(5)
+    # alpha = 0: g1 = g0, so phi(x) = exp(W_o W_s x + W_o b_s + b_o): the affine map `phi` with gamma = 0
+    P0 = dict(P, alpha=0.0)
+    want = O.phi(x, P["W_o"] @ P["W_s"], P["W_o"] @ P["b_s"] + P["b_o"], 0.0)
+    np.testing.assert_allclose(O.phi_mlp(x, **P0), want, rtol=1e-13)
+    # general alpha: scalar loops written out
+    emb, r = 7, 4
+    g0 = [sum(P["W_s"][i][c] * x[c] for c in range(5)) + P["b_s"][i] for i in range(emb)]
+    pre = [sum(P["W_1"][i][c] * g0[c] for c in range(emb)) + P["b_1"][i] for i in range(emb)]
+    h = [0.5 * t * (1 + math.erf(t / math.sqrt(2))) for t in pre]
+    delta = [sum(P["W_2"][i][c] * h[c] for c in range(emb)) + P["b_2"][i] for i in range(emb)]
+    g1 = [g0[i] + P["alpha"] * delta[i] for i in range(emb)]
+    out = [math.exp(sum(P["W_o"][j][c] * g1[c] for c in range(emb)) + P["b_o"][j]) for j in range(r)]
+    np.testing.assert_allclose(O.phi_mlp(x, **P), out, rtol=1e-13)
+    assert (O.phi_mlp(10 * g.standard_normal((6, 5)), **P) > 0).all()               # positivity by exponentiation
+    # rows are independent: the batch form equals the vector form
+    X = g.standard_normal((3, 5))
+    np.testing.assert_allclose(O.phi_mlp(X, **P)[1], O.phi_mlp(X[1], **P), rtol=1e-13)
+    # a transposed W_1 or a missing residual gives something else
+    assert np.abs(O.phi_mlp(x, **dict(P, W_1=P["W_1"].T)) - np.array(out)).max() > 1e-6
+
+
 def test_reassociated_form_equals_literal():
     p = _rand_problem(15)
     res = _run(p, 7)
