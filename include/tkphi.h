@@ -56,7 +56,7 @@ typedef enum {
 } tkphi_status;
 
 /* Which entry point a workspace is sized for. */
-enum { TKPHI_WS_BUILD = 0, TKPHI_WS_TOPK_DECODE = 1, TKPHI_WS_DECODE_STEP = 2 };
+enum { TKPHI_WS_BUILD = 0, TKPHI_WS_TOPK_DECODE = 1, TKPHI_WS_DECODE_STEP = 2, TKPHI_WS_MLP_KEY_FEATURES = 3 };
 
 /* Flags of tkphi_decode_step. */
 enum {
@@ -226,6 +226,56 @@ tkphi_status tkphi_decode_step(const tkphi_kv_desc* kv, const tkphi_phi_desc* ph
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The paper's own feature map (App. C.2, "Head-wise phi architecture"): a one-block ReZero MLP of
+ * hidden width d_emb per head,
+ *   g0 = W_s x + b_s;  Delta = W_2 GeLU(W_1 g0 + b_1) + b_2;  g1 = g0 + alpha Delta;  phi(x) = exp(W_o g1 + b_o),
+ * GeLU(t) = t Phi(t) with the normal CDF (erf form).  One descriptor holds the maps of one side:
+ * n_heads = n_q_heads for phi_q, n_kv_heads for phi_k.  Row-major fp32 device parameters, every
+ * pointer 16-byte aligned; d_emb a multiple of 128, at most 512.
+ */
+typedef struct {
+  int32_t d_emb, n_heads;
+  const float* w_s; const float* b_s; /* [n_heads][d_emb][head_dim], [n_heads][d_emb] */
+  const float* w_1; const float* b_1; /* [n_heads][d_emb][d_emb],    [n_heads][d_emb] */
+  const float* w_2; const float* b_2; /* [n_heads][d_emb][d_emb],    [n_heads][d_emb] */
+  const float* alpha;                 /* [n_heads] */
+  const float* w_o; const float* b_o; /* [n_heads][n_feat][d_emb],   [n_heads][n_feat] */
+} tkphi_mlp_desc;
+
+/*
+ * Key features of the MLP map (App. C.2) for a whole cache: phi_k(k_t) of EVERY cache row t of every
+ * KV head (anchor rows included) is written to phi_k_cache, fp32 [n_kv_heads][T_total][n_feat]
+ * (layout as in tkphi_phi_desc).  The four layers run as tensor-core GEMMs over all tokens with
+ * bf16 operands (weights and the activations between the layers are rounded to bf16), fp32
+ * accumulation, biases, residual and exponent.  Workspace: tkphi_workspace_bytes(kv, NULL, 0,
+ * TKPHI_WS_MLP_KEY_FEATURES).  Feed the cache to tkphi_build_summaries_cached and
+ * tkphi_decode_step_mlp.
+ */
+tkphi_status tkphi_mlp_key_features(const tkphi_kv_desc* kv, const tkphi_mlp_desc* mlp_k, float* phi_k_cache,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Prefill summary build (Sec. 4.1, Eq. natural_cache) from stored key features: S[b][h] = sum_{i in M_b}
+ * v_i phi_k(k_i)^T, u[b][h] = sum phi_k(k_i) with phi_k(k_i) read from row cu_seqlens[b] + i of
+ * phi_k_cache (as tkphi_mlp_key_features, or tkphi_build_summaries with a cache, wrote it).  kv->k is
+ * validated like every descriptor field (a valid device pointer) but its rows are not read.  Outputs, workspace (TKPHI_WS_BUILD) and errors as for tkphi_build_summaries.
+ */
+tkphi_status tkphi_build_summaries_cached(const tkphi_kv_desc* kv, const float* phi_k_cache, float* S, float* u,
+                                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Top-K+phi decode step (Sec. 4.2-4.3) with the paper's MLP feature maps (App. C.2): phi_q(q) is
+ * evaluated by the library from mlp_q (n_heads = n_q_heads), the retrieved keys' features are taken
+ * from phi_k_cache (the MLP is never re-evaluated for keys at decode time).  With TKPHI_FLAG_NOSUB the
+ * cache is not read and may be NULL.  Everything else as for tkphi_decode_step; workspace
+ * TKPHI_WS_DECODE_STEP.
+ */
+tkphi_status tkphi_decode_step_mlp(const tkphi_kv_desc* kv, const tkphi_mlp_desc* mlp_q, const float* phi_k_cache,
+                                   const void* q, const int32_t* topk_host, const int32_t* topk_dev, int32_t topk_max,
+                                   const float* S, const float* u, int32_t* idx_out, float* y_out, float* dbg_out,
+                                   uint32_t flags, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Reads the device status word that the kernels of the last call using this
  * workspace set (0 = fine; TKPHI_ERR_TIMEOUT if a bounded wait ran out).  Waits
  * for the stream.  *status_out is a host int.
@@ -262,7 +312,8 @@ enum {
   TKPHI_KERNEL_BUILD = 3,           /* prefill summary build */
   TKPHI_KERNEL_MEMSET = 4,          /* clearing counters when there is nothing to score */
   TKPHI_KERNEL_CACHED_Z = 5,        /* <phi_q, cached phi_k row> of the retrieved tokens (phi_k_cache given) */
-  TKPHI_KERNEL_KINDS = 6
+  TKPHI_KERNEL_MLP = 6,             /* the layers of the MLP key feature map (weight conversion included) */
+  TKPHI_KERNEL_KINDS = 7
 };
 void tkphi_kernel_timing_enable(int32_t on);
 tkphi_status tkphi_kernel_timing_read(float* ms_out, int32_t* count_out);

@@ -161,19 +161,21 @@ def phi_mlp_log(x, W_s, b_s, W_1, b_1, W_2, b_2, alpha, W_o, b_o) -> np.ndarray:
         g0 = W_s x + b_s;  Delta = W_2 GeLU(W_1 g0 + b_1) + b_2;  g1 = g0 + alpha Delta;
         phi(x) = exp(W_o g1 + b_o).
 
-    Rows of x are vectors.  W_s: [d_emb, d_h], W_1, W_2: [d_emb, d_emb], W_o: [d_phi, d_emb].
+    Rows of x are vectors; a single vector in gives a single vector out.
+    W_s: [d_emb, d_h], W_1, W_2: [d_emb, d_emb], W_o: [d_phi, d_emb].
     """
+    single = np.asarray(x).ndim == 1
     x = np.atleast_2d(np.asarray(x, F64))
     g0 = x @ np.asarray(W_s, F64).T + np.asarray(b_s, F64)
     delta = gelu(g0 @ np.asarray(W_1, F64).T + np.asarray(b_1, F64)) @ np.asarray(W_2, F64).T + np.asarray(b_2, F64)
     g1 = g0 + float(alpha) * delta
-    return g1 @ np.asarray(W_o, F64).T + np.asarray(b_o, F64)
+    out = g1 @ np.asarray(W_o, F64).T + np.asarray(b_o, F64)
+    return out[0] if single else out
 
 
 def phi_mlp(x, W_s, b_s, W_1, b_1, W_2, b_2, alpha, W_o, b_o) -> np.ndarray:
-    """phi(x) > 0 of the ReZero MLP feature map; a single vector in gives a single vector out."""
-    out = np.exp(phi_mlp_log(x, W_s, b_s, W_1, b_1, W_2, b_2, alpha, W_o, b_o))
-    return out[0] if np.asarray(x).ndim == 1 else out
+    """phi(x) > 0 of the ReZero MLP feature map."""
+    return np.exp(phi_mlp_log(x, W_s, b_s, W_1, b_1, W_2, b_2, alpha, W_o, b_o))
 
 
 def phi_mlp_param_count(d_h: int, d_phi: int, d_emb: int = 512, n_scalars: int = 2) -> int:

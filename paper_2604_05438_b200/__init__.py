@@ -9,6 +9,11 @@ from .binding import (  # noqa: F401
     TkphiError,
     KVCache,
     PhiMaps,
+    MlpMaps,
+    mlp_key_features,
+    build_summaries_cached,
+    decode_step_mlp,
+    WS_MLP_KEY_FEATURES,
     load_library,
     library_path,
     workspace_bytes,

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libtkphi.so")
 _lib = None
 
-WS_BUILD, WS_TOPK_DECODE, WS_DECODE_STEP = 0, 1, 2
+WS_BUILD, WS_TOPK_DECODE, WS_DECODE_STEP, WS_MLP_KEY_FEATURES = 0, 1, 2, 3
 FLAG_NONE, FLAG_NOSUB = 0, 1
 
 EXPORTED_SYMBOLS = (
@@ -22,9 +22,10 @@ EXPORTED_SYMBOLS = (
     "tkphi_kernel_timing_enable", "tkphi_kernel_timing_read",
     "tkphi_build_summaries_static", "tkphi_static_last_error", "tkphi_static_device_status",
     "tkphi_selftest_timeout",
+    "tkphi_mlp_key_features", "tkphi_build_summaries_cached", "tkphi_decode_step_mlp",
 )
 STATIC_SCRATCH_BYTES = 8 << 20
-KERNEL_KINDS = ("score", "select", "exact_residual", "build", "memset", "cached_z")
+KERNEL_KINDS = ("score", "select", "exact_residual", "build", "memset", "cached_z", "mlp")
 ERR_TIMEOUT = -5
 
 
@@ -45,6 +46,12 @@ class _KvDesc(C.Structure):
 class _PhiDesc(C.Structure):
     _fields_ = [("w_q", C.c_void_p), ("b_q", C.c_void_p), ("w_k", C.c_void_p), ("b_k", C.c_void_p),
                 ("gamma_q", C.c_float), ("gamma_k", C.c_float), ("phi_k_cache", C.c_void_p)]
+
+
+class _MlpDesc(C.Structure):
+    _fields_ = [("d_emb", C.c_int32), ("n_heads", C.c_int32), ("w_s", C.c_void_p), ("b_s", C.c_void_p),
+                ("w_1", C.c_void_p), ("b_1", C.c_void_p), ("w_2", C.c_void_p), ("b_2", C.c_void_p),
+                ("alpha", C.c_void_p), ("w_o", C.c_void_p), ("b_o", C.c_void_p)]
 
 
 def library_path() -> str:
@@ -80,6 +87,16 @@ def load_library():
     lib.tkphi_decode_step.argtypes = [C.POINTER(_KvDesc), C.POINTER(_PhiDesc), C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.tkphi_mlp_key_features.restype = C.c_int
+    lib.tkphi_mlp_key_features.argtypes = [C.POINTER(_KvDesc), C.POINTER(_MlpDesc), C.c_void_p, C.c_void_p, C.c_size_t,
+                                           C.c_void_p]
+    lib.tkphi_build_summaries_cached.restype = C.c_int
+    lib.tkphi_build_summaries_cached.argtypes = [C.POINTER(_KvDesc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                 C.c_size_t, C.c_void_p]
+    lib.tkphi_decode_step_mlp.restype = C.c_int
+    lib.tkphi_decode_step_mlp.argtypes = [C.POINTER(_KvDesc), C.POINTER(_MlpDesc), C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.tkphi_device_status.restype = C.c_int
     lib.tkphi_device_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
     lib.tkphi_kernel_timing_enable.restype = None
@@ -164,6 +181,27 @@ class PhiMaps:
                         float(self.gamma_q), float(self.gamma_k), cache)
 
 
+@dataclass
+class MlpMaps:
+    """fp32 device parameters of one side's ReZero-MLP feature maps (App. C.2): phi(x) =
+    exp(W_o (g0 + alpha (W_2 GeLU(W_1 g0 + b_1) + b_2)) + b_o), g0 = W_s x + b_s; leading dim = heads."""
+    w_s: torch.Tensor
+    b_s: torch.Tensor
+    w_1: torch.Tensor
+    b_1: torch.Tensor
+    w_2: torch.Tensor
+    b_2: torch.Tensor
+    alpha: torch.Tensor
+    w_o: torch.Tensor
+    b_o: torch.Tensor
+
+    def desc(self) -> _MlpDesc:
+        ts = (self.w_s, self.b_s, self.w_1, self.b_1, self.w_2, self.b_2, self.alpha, self.w_o, self.b_o)
+        for t in ts:
+            assert t.dtype == torch.float32 and t.is_contiguous()
+        return _MlpDesc(self.w_1.shape[1], self.w_s.shape[0], *[t.data_ptr() for t in ts])
+
+
 def _topk_host(topk) -> np.ndarray:
     return np.ascontiguousarray(topk, dtype=np.int32)
 
@@ -213,6 +251,35 @@ def selftest_timeout(workspace: torch.Tensor, stream=None) -> None:
     lib = load_library()
     _check(lib.tkphi_selftest_timeout(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                       _stream_ptr(stream)))
+
+
+def mlp_key_features(kv: KVCache, mlp_k: MlpMaps, phi_k_cache: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    lib = load_library()
+    d, m = kv.desc(), mlp_k.desc()
+    _check(lib.tkphi_mlp_key_features(C.byref(d), C.byref(m), phi_k_cache.data_ptr(), workspace.data_ptr(),
+                                      workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
+
+
+def build_summaries_cached(kv: KVCache, phi_k_cache: torch.Tensor, S: torch.Tensor, u: torch.Tensor,
+                           workspace: torch.Tensor, stream=None) -> None:
+    lib = load_library()
+    d = kv.desc()
+    _check(lib.tkphi_build_summaries_cached(C.byref(d), phi_k_cache.data_ptr(), S.data_ptr(), u.data_ptr(),
+                                            workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                            _stream_ptr(stream)))
+
+
+def decode_step_mlp(kv: KVCache, mlp_q: MlpMaps, phi_k_cache: Optional[torch.Tensor], q: torch.Tensor, topk_host,
+                    topk_dev: torch.Tensor, topk_max: int, S: torch.Tensor, u: torch.Tensor,
+                    idx_out: Optional[torch.Tensor], y_out: torch.Tensor, dbg_out: Optional[torch.Tensor], flags: int,
+                    workspace: torch.Tensor, stream=None) -> None:
+    lib = load_library()
+    d, m = kv.desc(), mlp_q.desc()
+    th = _topk_host(topk_host)
+    _check(lib.tkphi_decode_step_mlp(C.byref(d), C.byref(m), _ptr(phi_k_cache), q.data_ptr(), th.ctypes.data,
+                                     topk_dev.data_ptr(), int(topk_max), S.data_ptr(), u.data_ptr(), _ptr(idx_out),
+                                     y_out.data_ptr(), _ptr(dbg_out), int(flags), workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
 
 
 def topk_decode(kv: KVCache, q: torch.Tensor, topk_host, topk_dev: torch.Tensor, topk_max: int,

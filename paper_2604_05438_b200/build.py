@@ -10,7 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtkphi.so")
 SOURCES = ["api.cu", "score.cu", "select_cluster.cu", "exact_residual.cu", "build_summaries.cu", "static_scratch.cu",
-           "selftest.cu", "cached_features.cu"]
+           "selftest.cu", "cached_features.cu",
+           "mlp_features.cu"]
 HEADERS = ["common.cuh", "sm100.cuh", "feature_jobs.cuh", os.path.join("..", "..", "include", "tkphi.h")]
 
 

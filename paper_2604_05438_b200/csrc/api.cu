@@ -240,10 +240,67 @@ tkphi_status cuda_fail(cudaError_t e, const char* what) {
   return fail(TKPHI_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+// Workspace of tkphi_mlp_key_features: status word, bf16 copies of the weights, three bf16 activation
+// buffers [n_kv_heads][T_total][d_emb] (g0, GeLU output, g1).
+struct MlpLayout { size_t status, w_s, w_1, w_2, w_o, g0, h, g1, total; };
+MlpLayout mlp_layout(const tkphi_kv_desc* kv, const Shape& sh, int E) {
+  MlpLayout L{};
+  const size_t H = kv->n_kv_heads, T = (size_t)sh.total_tokens;
+  size_t o = 0;
+  L.status = o; o += 1024;
+  L.w_s = o;    o = align_up(o + H * E * kv->head_dim * 2, 1024);
+  L.w_1 = o;    o = align_up(o + H * E * E * 2, 1024);
+  L.w_2 = o;    o = align_up(o + H * E * E * 2, 1024);
+  L.w_o = o;    o = align_up(o + H * kv->n_feat * E * 2, 1024);
+  L.g0 = o;     o = align_up(o + H * T * E * 2, 1024);
+  L.h = o;      o = align_up(o + H * T * E * 2, 1024);
+  L.g1 = o;     o = align_up(o + H * T * E * 2, 1024);
+  L.total = o;
+  return L;
+}
+
+// 3-D view [head][row][k] of a bf16 matrix set for the MLP layers: box = 64 k x box_rows rows of one head,
+// 128-byte swizzle.  Strides in elements.
+tkphi_status make_gemm_map(const void* base, long long k, long long rows, long long heads, long long stride_row,
+                           long long stride_head, int box_rows, CUtensorMap* tm) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return fail(TKPHI_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  const cuuint64_t dims[3] = {(cuuint64_t)k, (cuuint64_t)rows, (cuuint64_t)heads};
+  cuuint64_t st[2] = {(cuuint64_t)stride_row * 2, (cuuint64_t)stride_head * 2};
+  if (heads == 1) st[1] = st[0] * (cuuint64_t)rows;
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, st, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(TKPHI_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return TKPHI_OK;
+}
+
+tkphi_status validate_mlp(const tkphi_mlp_desc* m, int n_heads, const char* what) {
+  if (!m) return fail(TKPHI_ERR_INVALID_ARG, "%s is NULL", what);
+  if (m->d_emb < 128 || m->d_emb > 512 || m->d_emb % 128 != 0)
+    return fail(TKPHI_ERR_UNSUPPORTED, "%s: d_emb must be 128, 256, 384 or 512, got %d", what, m->d_emb);
+  if (m->n_heads != n_heads) return fail(TKPHI_ERR_INVALID_ARG, "%s: n_heads = %d, expected %d", what, m->n_heads, n_heads);
+  const void* ptrs[9] = {m->w_s, m->b_s, m->w_1, m->b_1, m->w_2, m->b_2, m->alpha, m->w_o, m->b_o};
+  for (const void* q : ptrs)
+    if (!q || !aligned16(q)) return fail(TKPHI_ERR_INVALID_ARG, "%s: a parameter pointer is NULL or not 16-byte aligned", what);
+  return TKPHI_OK;
+}
+
+MlpParams mlp_params(const tkphi_mlp_desc* m) {
+  MlpParams o{};
+  o.d_emb = m->d_emb;
+  o.w_s = m->w_s; o.b_s = m->b_s; o.w_1 = m->w_1; o.b_1 = m->b_1; o.w_2 = m->w_2; o.b_2 = m->b_2;
+  o.alpha = m->alpha; o.w_o = m->w_o; o.b_o = m->b_o;
+  return o;
+}
+
 tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, const void* q,
                            const int32_t* topk_host, const int32_t* topk_dev, int32_t topk_max, const float* S,
                            const float* u, int32_t* idx_out, float* y_out, float* dbg_out, uint32_t flags,
-                           void* ws, size_t ws_bytes, void* stream, bool with_phi) {
+                           void* ws, size_t ws_bytes, void* stream, bool with_phi,
+                           const tkphi_mlp_desc* mlp_q = nullptr, const float* mlp_cache = nullptr) {
   g_err[0] = 0;
   Shape sh{};
   tkphi_status st = validate_kv(kv, &sh, true);
@@ -254,7 +311,13 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   if (!q || !aligned16(q)) return fail(TKPHI_ERR_INVALID_ARG, "q is NULL or not 16-byte aligned");
   if (!y_out) return fail(TKPHI_ERR_INVALID_ARG, "y_out is NULL");
   if (flags & ~1u) return fail(TKPHI_ERR_INVALID_ARG, "unknown flag bits 0x%x", flags);
-  if (with_phi) {
+  if (with_phi && mlp_q) {
+    st = validate_mlp(mlp_q, kv->n_q_heads, "mlp_q");
+    if (st != TKPHI_OK) return st;
+    if (!S || !u || !aligned16(S) || !aligned16(u)) return fail(TKPHI_ERR_INVALID_ARG, "S or u is NULL or not 16-byte aligned");
+    if (!(flags & TKPHI_FLAG_NOSUB) && (!mlp_cache || !aligned16(mlp_cache)))
+      return fail(TKPHI_ERR_INVALID_ARG, "phi_k_cache is NULL or not 16-byte aligned");
+  } else if (with_phi) {
     if (!phi || !phi->w_q || !phi->b_q || !phi->w_k || !phi->b_k)
       return fail(TKPHI_ERR_INVALID_ARG, "phi descriptor or one of its pointers is NULL");
     if (!S || !u) return fail(TKPHI_ERR_INVALID_ARG, "S or u is NULL");
@@ -281,7 +344,14 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   p.k = static_cast<const __nv_bfloat16*>(kv->k); p.v = static_cast<const __nv_bfloat16*>(kv->v);
   p.stride_head = kv->kv_stride_head; p.stride_token = kv->kv_stride_token;
   p.q = static_cast<const __nv_bfloat16*>(q);
-  if (with_phi) {
+  if (with_phi && mlp_q) {
+    p.mlp_q = mlp_params(mlp_q);
+    p.S = S; p.u = u;
+    if (!(flags & TKPHI_FLAG_NOSUB)) {
+      p.phi_cache = mlp_cache;
+      p.zbuf = reinterpret_cast<float*>(w + L.zbuf);
+    }
+  } else if (with_phi) {
     p.w_q = phi->w_q; p.b_q = phi->b_q; p.w_k = phi->w_k; p.b_k = phi->b_k;
     p.gamma_q = phi->gamma_q; p.gamma_k = phi->gamma_k; p.S = S; p.u = u;
     if (phi->phi_k_cache && !(flags & TKPHI_FLAG_NOSUB)) {
@@ -358,6 +428,45 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   return TKPHI_OK;
 }
 
+tkphi_status build_common(const tkphi_kv_desc* kv, const float* w_k, const float* b_k, float gamma_k, float* cache,
+                          bool from_cache, float* S, float* u, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  Shape sh{};
+  tkphi_status st = validate_kv(kv, &sh, true);
+  if (st != TKPHI_OK) return st;
+  if (!S || !u) return fail(TKPHI_ERR_INVALID_ARG, "S or u is NULL");
+  if (cache && !aligned16(cache)) return fail(TKPHI_ERR_INVALID_ARG, "phi_k_cache must be 16-byte aligned");
+  WsLayout L{};
+  build_layout(kv, sh, &L);
+  st = check_ws(workspace, workspace_bytes, L.total);
+  if (st != TKPHI_OK) return st;
+  cudaStream_t cs = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* w = static_cast<char*>(workspace);
+  BuildProblem p{};
+  p.batch = kv->batch; p.n_kv_heads = kv->n_kv_heads; p.head_dim = kv->head_dim; p.n_feat = kv->n_feat;
+  p.n_sink = kv->n_sink; p.n_tail = kv->n_tail;
+  p.cu_seqlens = reinterpret_cast<const long long*>(kv->cu_seqlens_dev);
+  p.k = static_cast<const __nv_bfloat16*>(kv->k); p.v = static_cast<const __nv_bfloat16*>(kv->v);
+  p.stride_head = kv->kv_stride_head; p.stride_token = kv->kv_stride_token;
+  p.w_k = w_k; p.b_k = b_k; p.gamma_k = gamma_k;
+  p.phi_cache = cache; p.from_cache = from_cache ? 1 : 0; p.total_tokens = sh.total_tokens;
+  p.S = S; p.u = u;
+  p.status = reinterpret_cast<int*>(w + L.status);
+  p.partials = reinterpret_cast<float*>(w + L.b_partials);
+  p.chunks_per_unit = L.chunks_per_unit;
+  CUtensorMap tk, tv;
+  st = make_tensor_map(kv, kv->k, 128, sh.total_tokens, &tk);
+  if (st != TKPHI_OK) return st;
+  st = make_tensor_map(kv, kv->v, 128, sh.total_tokens, &tv);
+  if (st != TKPHI_OK) return st;
+  cudaError_t e;
+  {
+    ScopedSpan sp(cs, TKPHI_KERNEL_BUILD);
+    e = launch_build(p, tk, tv, cs);      // clears the status word itself; needs no zeroed counters
+  }
+  if (e != cudaSuccess) return cuda_fail(e, "build launch");
+  return TKPHI_OK;
+}
+
 }  // namespace
 
 namespace tkphi {
@@ -401,6 +510,7 @@ size_t tkphi_workspace_bytes(const tkphi_kv_desc* kv, const int32_t* topk_host, 
     build_layout(kv, sh, &L);
     return L.total;
   }
+  if (which == TKPHI_WS_MLP_KEY_FEATURES) return mlp_layout(kv, sh, 512).total;
   if (which != TKPHI_WS_TOPK_DECODE && which != TKPHI_WS_DECODE_STEP) {
     fail(TKPHI_ERR_INVALID_ARG, "unknown workspace kind %d", which);
     return 0;
@@ -413,44 +523,77 @@ size_t tkphi_workspace_bytes(const tkphi_kv_desc* kv, const int32_t* topk_host, 
 tkphi_status tkphi_build_summaries(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, float* S, float* u,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
   g_err[0] = 0;
+  if (!phi || !phi->w_k || !phi->b_k) return fail(TKPHI_ERR_INVALID_ARG, "phi->w_k or phi->b_k is NULL");
+  if (!std::isfinite(phi->gamma_k)) return fail(TKPHI_ERR_INVALID_ARG, "gamma_k must be finite");
+  if (!aligned16(phi->w_k)) return fail(TKPHI_ERR_INVALID_ARG, "w_k must be 16-byte aligned");
+  return build_common(kv, phi->w_k, phi->b_k, phi->gamma_k, phi->phi_k_cache, false, S, u, workspace, workspace_bytes,
+                      cuda_stream);
+}
+
+tkphi_status tkphi_build_summaries_cached(const tkphi_kv_desc* kv, const float* phi_k_cache, float* S, float* u,
+                                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!phi_k_cache) return fail(TKPHI_ERR_INVALID_ARG, "phi_k_cache is NULL");
+  return build_common(kv, nullptr, nullptr, 0.f, const_cast<float*>(phi_k_cache), true, S, u, workspace, workspace_bytes,
+                      cuda_stream);
+}
+
+tkphi_status tkphi_mlp_key_features(const tkphi_kv_desc* kv, const tkphi_mlp_desc* mlp_k, float* phi_k_cache,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  g_err[0] = 0;
   Shape sh{};
   tkphi_status st = validate_kv(kv, &sh, true);
   if (st != TKPHI_OK) return st;
-  if (!phi || !phi->w_k || !phi->b_k) return fail(TKPHI_ERR_INVALID_ARG, "phi->w_k or phi->b_k is NULL");
-  if (!std::isfinite(phi->gamma_k)) return fail(TKPHI_ERR_INVALID_ARG, "gamma_k must be finite");
-  if (!S || !u) return fail(TKPHI_ERR_INVALID_ARG, "S or u is NULL");
-  WsLayout L{};
-  build_layout(kv, sh, &L);
+  st = validate_mlp(mlp_k, kv->n_kv_heads, "mlp_k");
+  if (st != TKPHI_OK) return st;
+  if (!phi_k_cache || !aligned16(phi_k_cache)) return fail(TKPHI_ERR_INVALID_ARG, "phi_k_cache is NULL or not 16-byte aligned");
+  const int E = mlp_k->d_emb, D = kv->head_dim, R = kv->n_feat, H = kv->n_kv_heads;
+  const long long T = sh.total_tokens;
+  const MlpLayout L = mlp_layout(kv, sh, E);
   st = check_ws(workspace, workspace_bytes, L.total);
   if (st != TKPHI_OK) return st;
   cudaStream_t cs = reinterpret_cast<cudaStream_t>(cuda_stream);
   char* w = static_cast<char*>(workspace);
-  BuildProblem p{};
-  p.batch = kv->batch; p.n_kv_heads = kv->n_kv_heads; p.head_dim = kv->head_dim; p.n_feat = kv->n_feat;
-  p.n_sink = kv->n_sink; p.n_tail = kv->n_tail;
-  p.cu_seqlens = reinterpret_cast<const long long*>(kv->cu_seqlens_dev);
-  p.k = static_cast<const __nv_bfloat16*>(kv->k); p.v = static_cast<const __nv_bfloat16*>(kv->v);
-  p.stride_head = kv->kv_stride_head; p.stride_token = kv->kv_stride_token;
-  p.w_k = phi->w_k; p.b_k = phi->b_k; p.gamma_k = phi->gamma_k;
-  p.phi_cache = phi->phi_k_cache; p.total_tokens = sh.total_tokens;
-  p.S = S; p.u = u;
-  p.status = reinterpret_cast<int*>(w + L.status);
-  p.partials = reinterpret_cast<float*>(w + L.b_partials);
-  p.chunks_per_unit = L.chunks_per_unit;
-  if (!aligned16(phi->w_k)) return fail(TKPHI_ERR_INVALID_ARG, "w_k must be 16-byte aligned");
-  if (phi->phi_k_cache && !aligned16(phi->phi_k_cache))
-    return fail(TKPHI_ERR_INVALID_ARG, "phi_k_cache must be 16-byte aligned");
-  CUtensorMap tk, tv;
-  st = make_tensor_map(kv, kv->k, 128, sh.total_tokens, &tk);
-  if (st != TKPHI_OK) return st;
-  st = make_tensor_map(kv, kv->v, 128, sh.total_tokens, &tv);
-  if (st != TKPHI_OK) return st;
-  cudaError_t e;
-  {
-    ScopedSpan sp(cs, TKPHI_KERNEL_BUILD);
-    e = launch_build(p, tk, tv, cs);      // clears the status word itself; needs no zeroed counters
-  }
-  if (e != cudaSuccess) return cuda_fail(e, "build launch");
+  int* status = reinterpret_cast<int*>(w + L.status);
+  __nv_bfloat16* ws_ = reinterpret_cast<__nv_bfloat16*>(w + L.w_s);
+  __nv_bfloat16* w1_ = reinterpret_cast<__nv_bfloat16*>(w + L.w_1);
+  __nv_bfloat16* w2_ = reinterpret_cast<__nv_bfloat16*>(w + L.w_2);
+  __nv_bfloat16* wo_ = reinterpret_cast<__nv_bfloat16*>(w + L.w_o);
+  __nv_bfloat16* g0 = reinterpret_cast<__nv_bfloat16*>(w + L.g0);
+  __nv_bfloat16* hb = reinterpret_cast<__nv_bfloat16*>(w + L.h);
+  __nv_bfloat16* g1 = reinterpret_cast<__nv_bfloat16*>(w + L.g1);
+  ScopedSpan sp(cs, TKPHI_KERNEL_MLP);
+  cudaError_t e = cudaMemsetAsync(status, 0, 256, cs);
+  if (e == cudaSuccess) e = launch_f32_to_bf16(mlp_k->w_s, ws_, (size_t)H * E * D, cs);
+  if (e == cudaSuccess) e = launch_f32_to_bf16(mlp_k->w_1, w1_, (size_t)H * E * E, cs);
+  if (e == cudaSuccess) e = launch_f32_to_bf16(mlp_k->w_2, w2_, (size_t)H * E * E, cs);
+  if (e == cudaSuccess) e = launch_f32_to_bf16(mlp_k->w_o, wo_, (size_t)H * R * E, cs);
+  if (e != cudaSuccess) return cuda_fail(e, "weight conversion launch");
+  // tensor maps: activations [head][token][k] (the keys through the cache's own strides), weights [head][n][k]
+  CUtensorMap a_k, a_g0, a_h, a_g1, m_ws, m_w1, m_w2, m_wo;
+  const int bn_o = R % 128 == 0 ? 128 : 64;
+  if ((st = make_tensor_map(kv, kv->k, 128, T, &a_k)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(g0, E, T, H, E, T * E, 128, &a_g0)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(hb, E, T, H, E, T * E, 128, &a_h)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(g1, E, T, H, E, T * E, 128, &a_g1)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(ws_, D, E, H, D, (long long)E * D, 128, &m_ws)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(w1_, E, E, H, E, (long long)E * E, 128, &m_w1)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(w2_, E, E, H, E, (long long)E * E, 128, &m_w2)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(wo_, E, R, H, E, (long long)R * E, bn_o, &m_wo)) != TKPHI_OK) return st;
+  GemmArgs g{};
+  g.M = (int)T; g.status = status;
+  // g0 = W_s x + b_s
+  g.N = E; g.K = D; g.epi = kEpiBias; g.bias = mlp_k->b_s; g.out = g0; g.out_head_stride = T * E;
+  if ((e = launch_mlp_gemm(a_k, m_ws, g, H, cs)) != cudaSuccess) return cuda_fail(e, "MLP stem launch");
+  // h = GeLU(W_1 g0 + b_1)
+  g.K = E; g.epi = kEpiGelu; g.bias = mlp_k->b_1; g.out = hb;
+  if ((e = launch_mlp_gemm(a_g0, m_w1, g, H, cs)) != cudaSuccess) return cuda_fail(e, "MLP layer 1 launch");
+  // g1 = g0 + alpha (W_2 h + b_2)
+  g.epi = kEpiResidual; g.bias = mlp_k->b_2; g.alpha = mlp_k->alpha; g.resid = g0; g.out = g1;
+  if ((e = launch_mlp_gemm(a_h, m_w2, g, H, cs)) != cudaSuccess) return cuda_fail(e, "MLP layer 2 launch");
+  // phi = exp(W_o g1 + b_o)
+  g.N = R; g.epi = kEpiExp; g.bias = mlp_k->b_o; g.out = phi_k_cache; g.out_head_stride = T * R;
+  if ((e = launch_mlp_gemm(a_g1, m_wo, g, H, cs)) != cudaSuccess) return cuda_fail(e, "MLP output layer launch");
   return TKPHI_OK;
 }
 
@@ -467,6 +610,15 @@ tkphi_status tkphi_decode_step(const tkphi_kv_desc* kv, const tkphi_phi_desc* ph
                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
   return decode_common(kv, phi, q, topk_host, topk_dev, topk_max, S, u, idx_out, y_out, dbg_out, flags, workspace,
                        workspace_bytes, cuda_stream, true);
+}
+
+tkphi_status tkphi_decode_step_mlp(const tkphi_kv_desc* kv, const tkphi_mlp_desc* mlp_q, const float* phi_k_cache,
+                                   const void* q, const int32_t* topk_host, const int32_t* topk_dev, int32_t topk_max,
+                                   const float* S, const float* u, int32_t* idx_out, float* y_out, float* dbg_out,
+                                   uint32_t flags, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!mlp_q) { g_err[0] = 0; return fail(TKPHI_ERR_INVALID_ARG, "mlp_q is NULL"); }
+  return decode_common(kv, nullptr, q, topk_host, topk_dev, topk_max, S, u, idx_out, y_out, dbg_out, flags, workspace,
+                       workspace_bytes, cuda_stream, true, mlp_q, phi_k_cache);
 }
 
 tkphi_status tkphi_device_status(const void* workspace, void* cuda_stream, int32_t* status_out) {

@@ -60,7 +60,9 @@ __device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[
       : "memory");
 }
 
-template <int D, bool CACHE>
+// MODE 0: features computed; 1: computed and also stored to the feature cache; 2: read from the
+// feature cache (no key tiles, no GEMM 1): for feature maps evaluated elsewhere (mlp_features.cu).
+template <int D, int MODE>
 __global__ void __launch_bounds__(kBuildThreads, 1)
 build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
              const BuildProblem p) {
@@ -80,6 +82,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   uint64_t* p_ready = d1_full + 2;         // [2]  features stored to tensor memory
   uint64_t* n_ready = p_ready + 2;         // [2]  key norms of the tile in shared memory
   uint64_t* d2_full = n_ready + 2;         // [1]  last GEMM 2 complete
+  uint64_t* g2_done = d2_full + 1;         // [2]  GEMM 2 of the tile that used this feature buffer is complete
   float* snorm = reinterpret_cast<float*>(bars + 32);        // [2][128]  -gamma log2e |k_t|^2, -inf if masked
   float* ucomb = snorm + 2 * 128;                            // [2][128]
   int* misc = reinterpret_cast<int*>(ucomb + 2 * 128);
@@ -118,11 +121,12 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
       mbar_init(&d1_full[s], 1); mbar_init(&p_ready[s], 8); mbar_init(&n_ready[s], 4);
     }
     mbar_init(d2_full, 1);
+    mbar_init(&g2_done[0], 1); mbar_init(&g2_done[1], 1);
     mbar_fence_init();
     *s_abort = 0;
   }
   if (warp == 1) tmem_alloc(s_tmem, kBuildTmemCols);
-  {
+  if (MODE != 2) {
     const float* W = p.w_k + (size_t)kvh * R * D;
     constexpr int CPR = D / 8;
     for (int i = tid; i < 128 * CPR; i += kBuildThreads) {
@@ -161,13 +165,16 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
       for (int it = 0; it < n_my && ok; ++it) {
         const int row = row0 + (t0 + it) * kBT;
         const int ks = it % KS, vs = it % VS;
-        ok = mbar_wait(&k_empty[ks], ((uint32_t)(it / KS) & 1u) ^ 1u, s_abort);
-        if (!ok) break;
-        mbar_expect_tx(&k_full[ks], C::TILE);
+        if (MODE != 2) {
+          ok = mbar_wait(&k_empty[ks], ((uint32_t)(it / KS) & 1u) ^ 1u, s_abort);
+          if (!ok) break;
+          mbar_expect_tx(&k_full[ks], C::TILE);
 #pragma unroll
-        for (int x = 0; x < BOXES; ++x)
-          tma_load_3d(kring + ks * C::TILE + x * C::BOX, &tmap_k, &k_full[ks], x * 64, row, kvh, pol);
+          for (int x = 0; x < BOXES; ++x)
+            tma_load_3d(kring + ks * C::TILE + x * C::BOX, &tmap_k, &k_full[ks], x * 64, row, kvh, pol);
+        }
         ok = mbar_wait(&v_empty[vs], ((uint32_t)(it / VS) & 1u) ^ 1u, s_abort);
+        if (!ok && MODE == 2) break;
         if (!ok) {
           // the key copy just issued must land before shared memory is released
           for (uint32_t w = 0; w < kWaitPolls; ++w) {
@@ -211,8 +218,12 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
           umma_ts(tmem_base + kColD2, tmem_base + lo_col, bd, idesc2, 1u);
         }
         tc_commit(&v_empty[vs]);
+        tc_commit(&g2_done[buf]);
       };
-      for (int it = 0; it < n_my && ok; ++it) {
+      if (MODE == 2) {
+        for (int it = 0; it + 1 < n_my && ok; ++it) gemm2(it);
+      }
+      for (int it = 0; MODE != 2 && it < n_my && ok; ++it) {
         const int buf = it & 1, ks = it % KS;
         // No wait for GEMM 2 of tile it-2, whose A operand lives where this accumulator goes:
         // MMAs issued by one thread execute in issue order, and the feature warps touch the
@@ -242,15 +253,20 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     const int quad = warp & 3;                     // tensor-memory lane quadrant
     const int h = (warp - 2) >> 2;                 // which 64 tokens of the tile
     const int j = quad * 32 + lane;                // feature
-    const float bj = j < R ? p.b_k[(size_t)kvh * R + j] * kLog2e : 0.f;
+    const float bj = (MODE != 2 && j < R) ? p.b_k[(size_t)kvh * R + j] * kLog2e : 0.f;
     float u_acc = 0.f;                             // sum of feature j over this thread's tokens
-    // optional cached features: row of mid token 0 of this head, column j
-    float* cache_j = (CACHE && j < R) ? p.phi_cache + ((size_t)kvh * p.total_tokens + (size_t)row0) * R + j : nullptr;
+    // feature cache (written in mode 1, read in mode 2): row of mid token 0 of this head, column j
+    float* cache_j = (MODE != 0 && j < R) ? p.phi_cache + ((size_t)kvh * p.total_tokens + (size_t)row0) * R + j : nullptr;
     bool ok = true;
     for (int it = 0; it < n_my && ok; ++it) {
       const int buf = it & 1;
       const uint32_t ph = (uint32_t)(it >> 1) & 1u;
-      ok = mbar_wait(&d1_full[buf], ph, s_abort) && mbar_wait(&n_ready[buf], ph, s_abort);
+      if (MODE == 2) {
+        // the feature buffer is free once GEMM 2 of tile it - 2 has read it; snorm says which tokens are in the mid-region
+        ok = mbar_wait(&n_ready[buf], ph, s_abort) && (it < 2 || mbar_wait(&g2_done[buf], ph ^ 1u, s_abort));
+      } else {
+        ok = mbar_wait(&d1_full[buf], ph, s_abort) && mbar_wait(&n_ready[buf], ph, s_abort);
+      }
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after_sync();
@@ -258,13 +274,20 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         float v[32];
-        tmem_ld_x32(tmem_addr(tmem_base, quad * 32, kColD1 + buf * 128 + h * 64 + c * 32), v);
-        tc_wait_ld();
+        if (MODE == 2) {
+          const int tok0 = (t0 + it) * kBT + h * 64 + c * 32;
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            v[e] = (cache_j != nullptr && sn[c * 32 + e] == 0.f) ? __ldcs(cache_j + (size_t)(tok0 + e) * R) : 0.f;
+        } else {
+          tmem_ld_x32(tmem_addr(tmem_base, quad * 32, kColD1 + buf * 128 + h * 64 + c * 32), v);
+          tc_wait_ld();
+        }
         uint32_t hi[16], lo[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-          const float f0 = ex2_approx(v[2 * e] + bj + sn[c * 32 + 2 * e]);
-          const float f1 = ex2_approx(v[2 * e + 1] + bj + sn[c * 32 + 2 * e + 1]);
+          const float f0 = MODE == 2 ? v[2 * e] : ex2_approx(v[2 * e] + bj + sn[c * 32 + 2 * e]);
+          const float f1 = MODE == 2 ? v[2 * e + 1] : ex2_approx(v[2 * e + 1] + bj + sn[c * 32 + 2 * e + 1]);
           u_acc += f0;
           u_acc += f1;
           const __nv_bfloat162 hp = __floats2bfloat162_rn(f0, f1);          // .x (low half) = even token
@@ -272,7 +295,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
               __floats2bfloat162_rn(f0 - __bfloat162float(hp.x), f1 - __bfloat162float(hp.y));
           hi[e] = *reinterpret_cast<const uint32_t*>(&hp);
           lo[e] = *reinterpret_cast<const uint32_t*>(&lp);
-          if (CACHE && cache_j) {
+          if (MODE == 1 && cache_j) {
             // one token per store: the 32 lanes of the warp write 32 consecutive features
             const int tok = (t0 + it) * kBT + h * 64 + c * 32 + 2 * e;
             if (tok < n_mid) __stcs(cache_j + (size_t)tok * R, f0);
@@ -314,14 +337,14 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     for (int it = 0; it < n_my && ok; ++it) {
       const int buf = it & 1, ks = it % KS;
       // snorm[buf] was last read by the feature warps for tile it-2: wait for their p_ready
-      ok = mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort) &&
+      ok = (MODE == 2 || mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort)) &&
            mbar_wait(&p_ready[buf], ((uint32_t)(it >> 1) & 1u) ^ 1u, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       const unsigned char* tile = kring + ks * C::TILE;
       float kn = 0.f;
 #pragma unroll
-      for (int c = 0; c < D / 8; ++c) {
+      for (int c = 0; MODE != 2 && c < D / 8; ++c) {
         const uint4 raw = *reinterpret_cast<const uint4*>(tile + (c >> 3) * C::BOX + swz128(t, c & 7));
         const unsigned w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -334,7 +357,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
       const bool valid = (t0 + it) * kBT + t < n_mid;
       snorm[buf * 128 + t] = valid ? -g2 * kn : -INFINITY;   // exp2(-inf) = 0 removes rows outside the mid-region
       __syncwarp();
-      if (lane == 0) { mbar_arrive(&n_ready[buf]); mbar_arrive(&k_empty[ks]); }
+      if (lane == 0) { mbar_arrive(&n_ready[buf]); if (MODE != 2) mbar_arrive(&k_empty[ks]); }
     }
   }
 
@@ -381,15 +404,15 @@ __global__ void __launch_bounds__(kRedThreads) build_reduce_kernel(const BuildPr
   }
 }
 
-template <int D, bool CACHE>
+template <int D, int MODE>
 static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, const CUtensorMap& tv,
                                   cudaStream_t st) {
   static PerDeviceFlag configured;
   const size_t smem = BuildCfg<D>::total;
-  cudaError_t e = set_max_dynamic_smem(configured, reinterpret_cast<const void*>(build_kernel<D, CACHE>), smem);
+  cudaError_t e = set_max_dynamic_smem(configured, reinterpret_cast<const void*>(build_kernel<D, MODE>), smem);
   if (e != cudaSuccess) return e;
   dim3 grid(p.chunks_per_unit, p.n_kv_heads, p.batch);
-  build_kernel<D, CACHE><<<grid, kBuildThreads, smem, st>>>(tk, tv, p);
+  build_kernel<D, MODE><<<grid, kBuildThreads, smem, st>>>(tk, tv, p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   // one output per thread: every thread's loads of all chunk partials are in flight at once
@@ -399,8 +422,11 @@ static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, 
 }
 
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tk, const CUtensorMap& tv, cudaStream_t st) {
-  if (p.head_dim == 64) return p.phi_cache ? launch_build_t<64, true>(p, tk, tv, st) : launch_build_t<64, false>(p, tk, tv, st);
-  if (p.head_dim == 128) return p.phi_cache ? launch_build_t<128, true>(p, tk, tv, st) : launch_build_t<128, false>(p, tk, tv, st);
+  const int mode = !p.phi_cache ? 0 : (p.from_cache ? 2 : 1);
+  if (p.head_dim == 64)
+    return mode == 0 ? launch_build_t<64, 0>(p, tk, tv, st) : mode == 1 ? launch_build_t<64, 1>(p, tk, tv, st) : launch_build_t<64, 2>(p, tk, tv, st);
+  if (p.head_dim == 128)
+    return mode == 0 ? launch_build_t<128, 0>(p, tk, tv, st) : mode == 1 ? launch_build_t<128, 1>(p, tk, tv, st) : launch_build_t<128, 2>(p, tk, tv, st);
   return cudaErrorInvalidValue;
 }
 

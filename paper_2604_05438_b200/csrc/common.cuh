@@ -21,6 +21,16 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kStatusOk = 0;
 constexpr int kStatusTimeout = -5;
 
+// Device pointers of one side's ReZero-MLP feature maps (App. C.2); w_s == nullptr: not used.
+struct MlpParams {
+  int d_emb;
+  const float* w_s; const float* b_s;      // [heads][d_emb][head_dim], [heads][d_emb]
+  const float* w_1; const float* b_1;      // [heads][d_emb][d_emb],   [heads][d_emb]
+  const float* w_2; const float* b_2;
+  const float* alpha;                      // [heads]
+  const float* w_o; const float* b_o;      // [heads][n_feat][d_emb],  [heads][n_feat]
+};
+
 // Everything the kernels need to know about one layer call.
 struct Problem {
   int batch, n_q_heads, n_kv_heads, head_dim, n_feat, n_sink, n_tail, group;
@@ -34,6 +44,7 @@ struct Problem {
   // feature maps
   const float* w_q; const float* b_q; const float* w_k; const float* b_k;
   float gamma_q, gamma_k;
+  MlpParams mlp_q;                 // query-side MLP maps (mlp_q.w_s != nullptr: used instead of w_q, b_q, gamma_q)
   // cached key features (optional): phi_k rows [n_kv_heads][total_tokens][n_feat], and where the
   // decode step keeps z_i = <phi_q, phi_k(k_i)> / exp(m_q) of the retrieved tokens: [rows][topk_max]
   const float* phi_cache; long long total_tokens;
@@ -68,7 +79,8 @@ struct BuildProblem {
   const __nv_bfloat16* v;
   long long stride_head, stride_token;
   const float* w_k; const float* b_k; float gamma_k;
-  float* phi_cache;                // optional: phi_k rows of the mid-region tokens are also written here
+  float* phi_cache;                // optional: phi_k rows of the mid-region tokens are also written here ...
+  int from_cache;                  // ... or, if set, read from here instead of being computed
   long long total_tokens;
   float* S; float* u;
   int* status;
@@ -189,6 +201,22 @@ cudaError_t launch_select(const Problem& p, int max_mid, int n_sm, cudaStream_t 
 cudaError_t launch_exact_residual(const Problem& p, const CUtensorMap& gk, const CUtensorMap& gv, long long n_pairs, int n_sm,
                                   cudaStream_t stream);
 cudaError_t launch_cached_z(const Problem& p, cudaStream_t stream);
+
+// One dense layer of the MLP feature map on the tensor cores (mlp_features.cu):
+// out[h][m][n] = epilogue(sum_k A[h][m][k] W[h][n][k] + bias[h][n]).
+enum { kEpiBias = 0, kEpiGelu = 1, kEpiResidual = 2, kEpiExp = 3 };
+struct GemmArgs {
+  int M, N, K;                         // rows, output columns, reduction length (K a multiple of 64)
+  int epi;
+  const float* bias;                   // [heads][N]
+  const float* alpha;                  // [heads] (kEpiResidual)
+  const __nv_bfloat16* resid;          // [heads][M][N] (kEpiResidual): out = resid + alpha (acc + bias)
+  void* out;                           // bf16 [heads][M][N], or fp32 for kEpiExp
+  long long out_head_stride;           // elements between heads of out (and of resid)
+  int* status;
+};
+cudaError_t launch_mlp_gemm(const CUtensorMap& map_a, const CUtensorMap& map_w, const GemmArgs& g, int heads, cudaStream_t stream);
+cudaError_t launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t stream);
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, cudaStream_t stream);
 
 }  // namespace tkphi

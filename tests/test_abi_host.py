@@ -100,6 +100,35 @@ def test_decode_step_and_build_validation(lib):
     assert lib.tkphi_device_status(None, None, None) == -1
 
 
+def test_mlp_entry_points_validate_their_arguments(lib):
+    d, cu = _desc([0, 400])
+    topk = np.array([3], np.int32)
+    mk = lambda **kw: B._MlpDesc(kw.get("E", 512), kw.get("H", 2), *[kw.get("p%d" % i, 0x100 * (i + 1)) for i in range(9)])
+    feats = lambda m, cache=0x9000, ws=0x10000, wsb=1 << 40: lib.tkphi_mlp_key_features(
+        C.byref(d), C.byref(m) if m is not None else None, cache, ws, wsb, None)
+    assert feats(None) == -1
+    assert feats(mk(E=96)) == -2 and feats(mk(E=640)) == -2          # hidden width: 128, 256, 384, 512
+    assert feats(mk(H=8)) == -1 and b"n_heads" in lib.tkphi_last_error()   # key side: one map per KV head
+    assert feats(mk(p3=0)) == -1 and feats(mk(p7=0x808)) == -1
+    assert feats(mk(), cache=0) == -1 and feats(mk(), cache=0x9004) == -1
+    assert feats(mk(), ws=0) == -3 and feats(mk(), wsb=4096) == -3
+    assert lib.tkphi_workspace_bytes(C.byref(d), None, 0, T.WS_MLP_KEY_FEATURES) > 3 * 2 * 400 * 512 * 2
+    # summary build from cached rows
+    assert lib.tkphi_build_summaries_cached(C.byref(d), 0, 0x7000, 0x8000, 0x10000, 1 << 40, None) == -1
+    assert lib.tkphi_build_summaries_cached(C.byref(d), 0x9004, 0x7000, 0x8000, 0x10000, 1 << 40, None) == -1
+    assert lib.tkphi_build_summaries_cached(C.byref(d), 0x9000, 0, 0x8000, 0x10000, 1 << 40, None) == -1
+    assert lib.tkphi_build_summaries_cached(C.byref(d), 0x9000, 0x7000, 0x8000, 0x10000, 16, None) == -3
+    # decode step with the MLP on the query side: one map per query head; the cache may be NULL only with NOSUB
+    step = lambda m, cache=0x9000, flags=0, wsb=1 << 40: lib.tkphi_decode_step_mlp(
+        C.byref(d), C.byref(m), cache, 0x4000, topk.ctypes.data, 0x6000, 3, 0x7000, 0x8000, None, 0x5000, None,
+        flags, 0x10000, wsb, None)
+    assert step(mk(H=2)) == -1
+    assert step(mk(H=8), cache=0) == -1 and b"phi_k_cache" in lib.tkphi_last_error()
+    assert step(mk(H=8), cache=0, flags=1, wsb=1000) == -3           # passes validation without a cache
+    assert step(mk(H=8), wsb=1000) == -3
+    assert step(mk(H=8, E=100)) == -2
+
+
 def test_workspace_sizes_scale_with_the_problem(lib):
     d1, c1 = _desc([0, 4096], n_q=32, n_kv=8)
     d2, c2 = _desc([0, 8192], n_q=32, n_kv=8)

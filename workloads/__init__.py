@@ -13,6 +13,8 @@ from .synthetic import (  # noqa: F401
     draw_seq_lens,
     make_layer_inputs,
     make_phi_params,
+    MlpPhiParams,
+    make_mlp_phi_params,
     budget_to_topk,
     bf16_round,
 )

@@ -154,6 +154,57 @@ def make_phi_params(cfg: WorkloadConfig, seed: int, kind: str = "baseline",
                      w_k.float().contiguous(), b_k.float().contiguous(), gq, gk, kind)
 
 
+@dataclass
+class MlpPhiParams:
+    """Parameters of one side's one-block ReZero-MLP feature maps (hidden width d_emb), fp32;
+    the leading dimension runs over the heads of that side."""
+
+    w_s: torch.Tensor   # [H, d_emb, d]
+    b_s: torch.Tensor   # [H, d_emb]
+    w_1: torch.Tensor   # [H, d_emb, d_emb]
+    b_1: torch.Tensor   # [H, d_emb]
+    w_2: torch.Tensor   # [H, d_emb, d_emb]
+    b_2: torch.Tensor   # [H, d_emb]
+    alpha: torch.Tensor  # [H]
+    w_o: torch.Tensor   # [H, r, d_emb]
+    b_o: torch.Tensor   # [H, r]
+
+    def to(self, device) -> "MlpPhiParams":
+        return MlpPhiParams(*[getattr(self, f).to(device) for f in
+                              ("w_s", "b_s", "w_1", "b_1", "w_2", "b_2", "alpha", "w_o", "b_o")])
+
+    def head(self, h: int) -> dict:
+        """float64 numpy arrays of head h, keyed like the feature map's symbols."""
+        return dict(W_s=self.w_s[h].double().numpy(), b_s=self.b_s[h].double().numpy(),
+                    W_1=self.w_1[h].double().numpy(), b_1=self.b_1[h].double().numpy(),
+                    W_2=self.w_2[h].double().numpy(), b_2=self.b_2[h].double().numpy(),
+                    alpha=float(self.alpha[h]), W_o=self.w_o[h].double().numpy(), b_o=self.b_o[h].double().numpy())
+
+
+def make_mlp_phi_params(cfg: WorkloadConfig, seed: int, side: str, d_emb: int = 512, device="cpu",
+                        bo_shift: Optional[torch.Tensor] = None) -> MlpPhiParams:
+    """Random-init ReZero-MLP feature maps for the query side (one per query head) or the key side
+    (one per KV head): weights ~ N(0, 1/fan_in), biases ~ N(0, 0.1^2), alpha ~ U(0.3, 0.7) (a trained
+    gate is not zero), output rows scaled by 1/2 so that the exponents stay within a few units.
+    An optional per-head shift is added to b_o."""
+    H = cfg.n_q_heads if side == "q" else cfg.n_kv_heads
+    d, r = cfg.head_dim, cfg.n_feat
+    g = _gen(seed * 104729 + (1 if side == "q" else 2), device)
+    rn = lambda *shape: torch.randn(*shape, generator=g, device=device)
+    w_s = rn(H, d_emb, d) / math.sqrt(d)
+    b_s = 0.1 * rn(H, d_emb)
+    w_1 = rn(H, d_emb, d_emb) / math.sqrt(d_emb)
+    b_1 = 0.1 * rn(H, d_emb)
+    w_2 = rn(H, d_emb, d_emb) / math.sqrt(d_emb)
+    b_2 = 0.1 * rn(H, d_emb)
+    alpha = 0.3 + 0.4 * torch.rand(H, generator=g, device=device)
+    w_o = 0.5 * rn(H, r, d_emb) / math.sqrt(d_emb)
+    b_o = 0.1 * rn(H, r)
+    if bo_shift is not None:
+        b_o = b_o + bo_shift.to(device=device, dtype=torch.float32).reshape(-1, 1)
+    return MlpPhiParams(*[t.float().contiguous() for t in (w_s, b_s, w_1, b_1, w_2, b_2, alpha, w_o, b_o)])
+
+
 def draw_seq_lens(cfg: WorkloadConfig, seed: int) -> List[int]:
     """Prefill lengths of the workload's sequences: uniform in [seq_len_min, seq_len] for ragged
     workloads (the same for every layer of a seed), else seq_len for all."""
