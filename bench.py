@@ -29,7 +29,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from workloads import CONFIGS, make_layer_inputs, make_phi_params  # noqa: E402
+from workloads import CONFIGS, make_layer_inputs, make_mlp_phi_params, make_phi_params  # noqa: E402
 
 
 def _peaks():
@@ -140,12 +140,17 @@ def run_ours(args, rank, world, device):
     for l in range(n_layers):
         inp = make_layer_inputs(cfg, seed, layer=l, device=device,
                                 seq_lens=([N] * cfg.batch) if (args.seq_len or cfg.seq_len_min is None) else None, n_steps=1)
-        phi = make_phi_params(cfg, seed + l, device=device)
         kv = T.KVCache(inp.k, inp.v, inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, cfg.n_sink, cfg.n_tail)
         layers.append((inp, kv))
         cache = (torch.empty(cfg.n_kv_heads, int(inp.cu_seqlens[-1]), cfg.n_feat, device=device)
-                 if args.phi_cache else None)        # written by the build, read by the decode steps
-        phis.append(T.PhiMaps(phi.w_q, phi.b_q, phi.w_k, phi.b_k, phi.gamma_q, phi.gamma_k, cache))
+                 if (args.phi_cache or args.mlp_phi) else None)   # written by the build, read by the decode steps
+        if args.mlp_phi:      # the ReZero-MLP maps: (query side, key side, cache)
+            mq, mk = (make_mlp_phi_params(cfg, seed + l, side, device=device) for side in ("q", "k"))
+            phis.append((T.MlpMaps(mq.w_s, mq.b_s, mq.w_1, mq.b_1, mq.w_2, mq.b_2, mq.alpha, mq.w_o, mq.b_o),
+                         T.MlpMaps(mk.w_s, mk.b_s, mk.w_1, mk.b_1, mk.w_2, mk.b_2, mk.alpha, mk.w_o, mk.b_o), cache))
+        else:
+            phi = make_phi_params(cfg, seed + l, device=device)
+            phis.append(T.PhiMaps(phi.w_q, phi.b_q, phi.w_k, phi.b_k, phi.gamma_q, phi.gamma_k, cache))
     torch.cuda.synchronize()
     t_gen = time.time() - t_gen
     topk = layers[0][0].topk(args.budget)
@@ -161,11 +166,27 @@ def run_ours(args, rank, world, device):
         Ss.append(torch.empty(B, Hkv, d, r, device=device))
         us.append(torch.empty(B, Hkv, r, device=device))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    T.build_summaries(layers[0][1], phis[0], Ss[0], us[0], wsb)      # warm-up
+    mlp_ms = None
+    if args.mlp_phi:      # key features of every cache row first (timed by itself), then the build from those rows
+        wsm = torch.empty(T.workspace_bytes(kv0, None, 0, T.WS_MLP_KEY_FEATURES), dtype=torch.uint8, device=device)
+        T.mlp_key_features(layers[0][1], phis[0][1], phis[0][2], wsm)    # warm-up
+        torch.cuda.synchronize()
+        e0.record()
+        for l in range(n_layers):
+            T.mlp_key_features(layers[l][1], phis[l][1], phis[l][2], wsm)
+        e1.record()
+        torch.cuda.synchronize()
+        mlp_ms = e0.elapsed_time(e1)
+        assert T.device_status(wsm) == 0, "a device-side wait timed out"
+        del wsm
+        build_one = lambda l: T.build_summaries_cached(layers[l][1], phis[l][2], Ss[l], us[l], wsb)
+    else:
+        build_one = lambda l: T.build_summaries(layers[l][1], phis[l], Ss[l], us[l], wsb)
+    build_one(0)                                                     # warm-up
     torch.cuda.synchronize()
     e0.record()
     for l in range(n_layers):
-        T.build_summaries(layers[l][1], phis[l], Ss[l], us[l], wsb)
+        build_one(l)
     e1.record()
     torch.cuda.synchronize()
     build_ms = e0.elapsed_time(e1)
@@ -184,8 +205,12 @@ def run_ours(args, rank, world, device):
 
     def step(qs):
         for l in range(n_layers):
-            T.decode_step(layers[l][1], phis[l], qs[l], topk, topk_dev, tmax, Ss[l], us[l], None, y_dev[l],
-                          None, 0, ws)
+            if args.mlp_phi:
+                T.decode_step_mlp(layers[l][1], phis[l][0], phis[l][2], qs[l], topk, topk_dev, tmax, Ss[l], us[l],
+                                  None, y_dev[l], None, 0, ws)
+            else:
+                T.decode_step(layers[l][1], phis[l], qs[l], topk, topk_dev, tmax, Ss[l], us[l], None, y_dev[l],
+                              None, 0, ws)
 
     def barrier():
         torch.cuda.synchronize()
@@ -247,14 +272,15 @@ def run_ours(args, rank, world, device):
         "dtype": "bf16 K/V, f32 accumulate", "data": "synthetic",
         "config": {"workload": workload_string(cfg, n_layers, N, args.budget, tmax, seq_lens),
                    "l2": "inputs (K/V of all layers) exceed L2 by >100x; no flush needed",
-                   "replicas": world, "seed": seed, "phi_k_cache": bool(args.phi_cache)},
+                   "replicas": world, "seed": seed, "phi_k_cache": bool(args.phi_cache or args.mlp_phi),
+                   "phi": "one-block ReZero MLP, d_emb 512" if args.mlp_phi else "exp(Wx + b - |x|^2/2)"},
         "step_us": {"median": statistics.median(per_step) * 1e3, "min": min(per_step) * 1e3,
                     "max": max(per_step) * 1e3},
         "achieved_gbs": ab["total"] / (ms * 1e-3) / 1e9,
         "hbm_frac_of_measured_peak": ab["total"] / (ms * 1e-3) / 1e9 / peak,
         "algorithmic_bytes_per_step": ab["total"],
         "steps_per_s_all_gpus": whole_job_steps_per_s(ms, world),
-        "gpu_launches": args.steps * n_layers * (4 if args.phi_cache else 3),
+        "gpu_launches": args.steps * n_layers * (4 if (args.phi_cache or args.mlp_phi) else 3),
         "e2e": {"value": e2e_ms * 1e3, "unit": "us/step", "h2d_bytes_per_step": q_stage.numel() * 2,
                 "d2h_bytes_per_step": y_host.numel() * 4},
         "build": build_info(build_ms, n_layers, Hkv, sum(max(0, n - cfg.n_sink - cfg.n_tail) for n in seq_lens), d, r,
@@ -262,6 +288,11 @@ def run_ours(args, rank, world, device):
         "clocks": clocks,
         "gen_s": t_gen,
     }
+    if mlp_ms is not None:      # four GEMMs per token and KV head: d x E, E x E twice, E x r (E = hidden width 512)
+        E = 512
+        fl = 2.0 * n_layers * Hkv * sum(seq_lens) * (d * E + 2 * E * E + E * r)
+        out["mlp_key_features"] = {"ms_all_layers": mlp_ms, "tflops_bf16": fl / (mlp_ms * 1e-3) / 1e12,
+                                   "frac_of_bf16_sustained_peak": fl / (mlp_ms * 1e-3) / 1e12 / tf_sust}
     if kt is not None:
         dom = kt["score"]
         a = ab["key_stream_per_layer"] / (dom["avg_ms"] * 1e-3) / 1e9
@@ -392,6 +423,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--seq-len", type=int, default=0, help="override the context length (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mlp-phi", action="store_true",
+                    help="feature maps = the one-block ReZero MLP: key features by tkphi_mlp_key_features into a cache, "
+                         "summaries built from the cache, decode steps through tkphi_decode_step_mlp")
     ap.add_argument("--phi-cache", action="store_true",
                     help="keep the key features the build computes and read them at decode time (Sec. 4.2, cached variant)")
     args = ap.parse_args()

@@ -29,19 +29,24 @@ def _maps(T, p):
     return T.MlpMaps(p.w_s, p.b_s, p.w_1, p.b_1, p.w_2, p.b_2, p.alpha, p.w_o, p.b_o)
 
 
-def _calibrate_bo_shift(cfg, inp, pk, pq, frac, n_probe=2):
+def _log_features(X, params, chunk=16384):
+    """Oracle log phi(x) of the rows of X, a block of rows at a time (bounds the float64 intermediates)."""
+    return np.concatenate([O.phi_mlp_log(X[i:i + chunk], **params) for i in range(0, X.shape[0], chunk)], axis=0)
+
+
+def _calibrate_bo_shift(cfg, inp, pk, pq, frac, kv_heads, n_probe=2):
     """Per-KV-head shift of the key side's b_o that puts median(log Z_hat_R - log Z_R) at zero, so that
     the residual branch carries a visible share of the mass (oracle only, sequence 0)."""
     shift = torch.zeros(cfg.n_kv_heads)
     topk = int(inp.topk(frac)[0])
-    for kvh in range(cfg.n_kv_heads):
+    for kvh in kv_heads:
         K, V = PU.seq_arrays(inp, 0, kvh)
-        Phi = O.phi_mlp(K, **pk.head(kvh))
+        Phi = np.exp(_log_features(K, pk.head(kvh)))
         S, u = O.build_summaries_from_features(V, Phi, inp.n_sink, inp.n_tail)
         errs = []
         for n in range(n_probe):
             hq = kvh * cfg.group + n % cfg.group
-            q64 = inp.q[0, 0, hq].double().numpy()
+            q64 = inp.q[0, 0, hq].cpu().double().numpy()
             ret = O.select_topk(q64, K, inp.n_sink, inp.n_tail, topk)
             res = O.merge_from_features(q64, K, V, inp.n_sink, inp.n_tail, ret, S, u,
                                         O.phi_mlp_log(q64, **pq.head(hq)), Phi[ret])
@@ -52,13 +57,16 @@ def _calibrate_bo_shift(cfg, inp, pk, pq, frac, n_probe=2):
     return shift
 
 
-def _check_mlp(cfg, seed, seq_lens, frac, heads, d_emb=512):
+def _check_mlp(cfg, seed, seq_lens, frac, heads, d_emb=512, on_device=False):
+    """heads: the query heads compared; the oracle runs on their KV heads only."""
     import paper_2604_05438_b200 as T
     dev = torch.device("cuda:0")
-    inp = make_layer_inputs(cfg, seed, seq_lens=seq_lens, n_steps=1)
+    inp = make_layer_inputs(cfg, seed, seq_lens=seq_lens, n_steps=1, device=dev if on_device else "cpu")
+    heads = list(heads)
+    kv_heads = sorted({hq // cfg.group for hq in heads})
     pq = make_mlp_phi_params(cfg, seed, "q", d_emb)
     pk = make_mlp_phi_params(cfg, seed, "k", d_emb)
-    pk = make_mlp_phi_params(cfg, seed, "k", d_emb, bo_shift=_calibrate_bo_shift(cfg, inp, pk, pq, frac))
+    pk = make_mlp_phi_params(cfg, seed, "k", d_emb, bo_shift=_calibrate_bo_shift(cfg, inp, pk, pq, frac, kv_heads))
     kv = T.KVCache(inp.k.to(dev), inp.v.to(dev), inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, inp.n_sink, inp.n_tail)
     Hq, Hkv, d, r, B = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_feat, inp.batch
     T_total = int(inp.cu_seqlens[-1])
@@ -70,12 +78,11 @@ def _check_mlp(cfg, seed, seq_lens, frac, heads, d_emb=512):
     T.mlp_key_features(kv, _maps(T, pk.to(dev)), cache, ws)
     torch.cuda.synchronize()
     assert T.device_status(ws) == 0
-    ch = cache.cpu().double().numpy()
-    assert np.isfinite(ch).all() and (ch > 0).all()
+    assert bool(torch.isfinite(cache).all()) and bool((cache > 0).all())
+    ch = {kvh: cache[kvh].cpu().double().numpy() for kvh in kv_heads}
     Phi_o = {}
-    for kvh in range(Hkv):
-        K_all = inp.k[kvh].double().numpy()
-        a = O.phi_mlp_log(K_all, **pk.head(kvh))
+    for kvh in kv_heads:
+        a = _log_features(inp.k[kvh].cpu().double().numpy(), pk.head(kvh))
         Phi_o[kvh] = a
         e = np.abs(np.log(ch[kvh]) - a).max()
         assert PU.note("mlp_key_log_feature_abs_err", e) <= MLP_LOG_TOL, (kvh, e)
@@ -90,9 +97,9 @@ def _check_mlp(cfg, seed, seq_lens, frac, heads, d_emb=512):
     Sh, uh = S.cpu().double().numpy(), u.cpu().double().numpy()
     for b in range(B):
         lo, hi = int(inp.cu_seqlens[b]), int(inp.cu_seqlens[b + 1])
-        for kvh in range(Hkv):
+        for kvh in kv_heads:
             K, V = PU.seq_arrays(inp, b, kvh)
-            S0, u0 = O.build_summaries_from_features(V, ch[kvh, lo:hi], inp.n_sink, inp.n_tail)
+            S0, u0 = O.build_summaries_from_features(V, ch[kvh][lo:hi], inp.n_sink, inp.n_tail)
             if np.abs(S0).max() >= PU.FP32_TINY:
                 assert PU.note("S_rel_err", PU.max_rel(Sh[b, kvh], S0)) <= PU.SU_TOL, (b, kvh)
                 assert PU.note("u_rel_err", PU.max_rel(uh[b, kvh], u0)) <= PU.SU_TOL, (b, kvh)
@@ -127,11 +134,11 @@ def _check_mlp(cfg, seed, seq_lens, frac, heads, d_emb=512):
         for hq in heads:
             kvh = hq // cfg.group
             K, V = PU.seq_arrays(inp, b, kvh)
-            q64 = inp.q[0, b, hq].double().numpy()
+            q64 = inp.q[0, b, hq].cpu().double().numpy()
             kk = int(topk[b])
             ret = PU.check_selection(q64, K, inp.n_sink, inp.n_tail, kk, ih[b, hq])
             a_q = O.phi_mlp_log(q64, **pq.head(hq))
-            Phi_ret = ch[kvh, lo:hi][ret]
+            Phi_ret = ch[kvh][lo:hi][ret]
             res = O.merge_from_features(q64, K, V, inp.n_sink, inp.n_tail, ret, Sh[b, kvh], uh[b, kvh], a_q, Phi_ret)
             nosub = O.merge_from_features(q64, K, V, inp.n_sink, inp.n_tail, ret, Sh[b, kvh], uh[b, kvh], a_q, Phi_ret,
                                           subtract=False)
@@ -163,3 +170,9 @@ def test_mlp_phi_smaller_hidden_width_and_short_sequences():
     # d_emb = 256; a sequence with an empty mid-region contributes zero summaries
     cfg = dataclasses.replace(CONFIGS["c1_1b_4k"], n_tail=16)
     _check_mlp(cfg, 5, [700, 18, 129], 0.05, heads=range(0, cfg.n_q_heads, 3), d_emb=256)
+
+
+def test_mlp_phi_one_full_size_128k_layer_sampled_heads():
+    # one layer of the 128K workload in its own geometry and anchors; the oracle runs on two KV heads
+    cfg = CONFIGS["c3_3b_128k"]
+    _check_mlp(cfg, 0, None, 0.01, heads=[3, 4, 5, 21], on_device=True)
