@@ -3,23 +3,34 @@
 //   phi_k(k) = exp(W_k k + b_k - gamma_k |k|^2).
 //
 // Both contractions of the build are dense, so both run on the tensor cores
-// (tcgen05.mma, accumulators in tensor memory).  Per tile of 128 mid-region tokens:
+// (tcgen05.mma, accumulators in tensor memory).  Everything but the key and value tiles lives
+// in tensor memory, so that shared memory -- whose bandwidth the MMA operand reads, the TMA
+// writes and the norm reads share -- carries each tile only as often as it must, and all of
+// it is left to the key/value stream.  Per tile of 128 mid-region tokens:
 //   GEMM 1   A^T[j][t] = sum_c W_k[j][c] k_t[c]      A operand: W_k (split into bf16
-//            hi + lo, rows = features, zero padded to 128), B operand: the key tile as
-//            TMA lands it.  The fp32 result sits in tensor memory with one feature per
-//            lane and one token per column.
+//            hi + lo, rows = features, zero padded to 128) from tensor memory, B operand:
+//            the key tile as TMA lands it.  The fp32 result sits in tensor memory with one
+//            feature per lane and one token per column.
 //   features Phi^T[j][t] = exp2(A^T + b_j - gamma |k_t|^2) (everything pre-scaled by
-//            log2 e).  Eight warps read the accumulator, add u_j += Phi (fp32), split
-//            Phi into bf16 hi + lo (error ~2^-17) and store both back to tensor memory.
-//   GEMM 2   S^T[j][c] += sum_t Phi^T[j][t] v_t[c]   A operand: Phi^T hi, then lo,
-//            straight from tensor memory; B operand: the value tile as TMA lands it
-//            (tokens along K, dims contiguous).  S^T accumulates in tensor memory over
-//            all tiles of the CTA.
+//            log2 e).  Eight warps read the accumulator into registers, add u_j += Phi
+//            (fp32), split Phi into bf16 hi + lo (error ~2^-17) and store both over the
+//            accumulator columns they have read, as A operands (two tokens per column).
+//            There are two such accumulator / operand buffers, used by alternate tiles.
+//   GEMM 2   S^T[j][c] += sum_t Phi^T[j][t] v_t[c]   A operand: Phi^T hi, then lo, from
+//            tensor memory; B operand: the value tile as TMA lands it (MN-major: dims
+//            contiguous, tokens along K).  S^T accumulates in tensor memory over all tiles
+//            of the CTA.
+// (Stacking hi and lo along N, with the features passing through shared memory, was measured:
+// an MMA with N = 256 takes twice as long as one with N = 128, and the extra shared-memory
+// traffic slowed every MMA down.)
 // With a feature cache (Sec. 4.2 notes that a cached implementation avoids the decode-side
 // recompute) the feature warps also write every phi_k row they produce to global memory.
-// Warp roles: 0 TMA producer, 1 MMA issuer, 2..9 feature warps, 10..13 key norms.
-// GEMM 1 of tile i+1 is issued before GEMM 2 of tile i, so the tensor pipe works while
-// the feature warps are busy.  Each CTA owns a contiguous range of tiles of one
+// Warp roles: 0 TMA producer, 1 GEMM-1 issuer, then the feature warps, four key-norm warps, the GEMM-2 issuer (an
+// issuing thread advances only as fast as its MMAs execute, so with one issuer every barrier wait between
+// the two GEMMs of a tile was idle time of the tensor pipe).
+// Key and value tiles share one ring of shared-memory slots, filled in the order in which the
+// tensor pipe consumes them.  GEMM 1 of tile i+1 runs into the other buffer while the feature
+// warps work on tile i, so the tensor pipe works while the feature warps are busy.  Each CTA owns a contiguous range of tiles of one
 // (sequence, KV head) unit and writes one partial; a second small kernel adds the
 // partials in chunk order.  Every device-side wait is bounded and reports through the
 // status word.
@@ -28,28 +39,18 @@
 
 namespace tkphi {
 
-constexpr int kBuildThreads = 448;
+constexpr int kFWarps = 16;              // feature warps: four per tensor-memory lane quadrant
+constexpr int kTPT = 128 * 4 / kFWarps;  // tokens of a tile per feature thread (its feature, a contiguous token group)
+constexpr int kNG = kFWarps / 4;         // token groups of a tile
+constexpr int kWarpNorm = 2 + kFWarps;   // first of the four norm warps
+constexpr int kWarpG2 = kWarpNorm + 4;   // GEMM-2 issuer
+constexpr int kBuildThreads = (kWarpG2 + 1) * 32;
 constexpr int kBT = 128;                 // tokens per tile
 constexpr int kBuildTmemCols = 512;
-constexpr int kColD1 = 0;                // two GEMM-1 accumulators of 128 columns (Phi hi overwrites them)
-constexpr int kColD2 = 256;              // S^T accumulator, head_dim columns
-constexpr int kColLo = 384;              // Phi lo, 64 columns per buffer
-
-template <int D>
-struct BuildCfg {
-  static constexpr int BOXES = D / 64;
-  static constexpr int BOX = kBT * 128;                    // bytes of one 64-dim column block of a tile
-  static constexpr int TILE = BOXES * BOX;                 // 32 KB (d = 128) or 16 KB (d = 64)
-  static constexpr int KS = D == 128 ? 2 : 3;              // key ring stages
-  static constexpr int VS = D == 128 ? 2 : 3;              // value ring stages
-  static constexpr size_t whi = 0;
-  static constexpr size_t wlo = whi + TILE;
-  static constexpr size_t kring = wlo + TILE;
-  static constexpr size_t vring = kring + (size_t)KS * TILE;
-  static constexpr size_t small = vring + (size_t)VS * TILE;
-  // small: barriers (<= 32), snorm[2][128], ucomb[2][128], misc
-  static constexpr size_t total = small + 32 * 8 + 4 * (2 * 128 + 2 * 128 + 16);
-};
+constexpr int kColW = 0;                 // W_k as the A operand of GEMM 1: 64 packed columns hi, then 64 lo
+constexpr int kColBuf = 128;             // two buffers of 128 columns: GEMM-1 accumulator, then Phi^T hi / lo as the A operand
+                                         // of GEMM 2 (per token group of a feature thread: its packed columns hi, then lo)
+constexpr int kColD2 = 384;              // S^T accumulator, head_dim columns
 
 __device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
@@ -60,6 +61,18 @@ __device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[
       : "memory");
 }
 
+template <int D>
+struct BuildCfg {
+  static constexpr int BOXES = D / 64;
+  static constexpr int BOX = kBT * 128;                    // bytes of one 64-dim column block of a tile
+  static constexpr int TILE = BOXES * BOX;                 // 32 KB (d = 128) or 16 KB (d = 64)
+  static constexpr int NS = D == 128 ? 7 : 10;             // slots of the key/value ring (2 NS + 10 barriers <= 32)
+  static constexpr size_t ring = 0;
+  static constexpr size_t small = ring + (size_t)NS * TILE;
+  // small: barriers (<= 32), snorm[2][128], misc; the per-group feature sums reuse the ring at the end
+  static constexpr size_t total = small + 32 * 8 + 4 * (2 * 128 + 16);
+};
+
 // MODE 0: features computed; 1: computed and also stored to the feature cache; 2: read from the
 // feature cache (no key tiles, no GEMM 1): for feature maps evaluated elsewhere (mlp_features.cu).
 template <int D, int MODE>
@@ -67,25 +80,22 @@ __global__ void __launch_bounds__(kBuildThreads, 1)
 build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
              const BuildProblem p) {
   using C = BuildCfg<D>;
-  constexpr int KS = C::KS, VS = C::VS, BOXES = C::BOXES;
+  constexpr int NS = C::NS, BOXES = C::BOXES;
+  constexpr int LPT = MODE == 2 ? 1 : 2;       // ring loads per tile
   extern __shared__ __align__(1024) unsigned char smem[];
-  unsigned char* whi = smem + C::whi;
-  unsigned char* wlo = smem + C::wlo;
-  unsigned char* kring = smem + C::kring;
-  unsigned char* vring = smem + C::vring;
+  unsigned char* ring = smem + C::ring;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::small);
-  uint64_t* k_full = bars;                 // [KS] key tile landed
-  uint64_t* k_empty = k_full + KS;         // [KS] GEMM 1 and the norm warps are done with it
-  uint64_t* v_full = k_empty + KS;         // [VS]
-  uint64_t* v_empty = v_full + VS;         // [VS] GEMM 2 is done with it
-  uint64_t* d1_full = v_empty + VS;        // [2]  GEMM 1 accumulator complete
-  uint64_t* p_ready = d1_full + 2;         // [2]  features stored to tensor memory
+  uint64_t* full = bars;                   // [NS] tile landed
+  uint64_t* empty = full + NS;             // [NS] the MMAs that read the slot are complete (and, for a key tile, its norms taken)
+  uint64_t* d1_full = empty + NS;          // [2]  GEMM 1 accumulator complete
+  uint64_t* buf_free = d1_full + 2;        // [2]  GEMM 2 of the tile is complete: its buffer may take the next accumulator
+  uint64_t* p_ready = buf_free + 2;        // [2]  feature operand of the tile stored to tensor memory
   uint64_t* n_ready = p_ready + 2;         // [2]  key norms of the tile in shared memory
   uint64_t* d2_full = n_ready + 2;         // [1]  last GEMM 2 complete
-  uint64_t* g2_done = d2_full + 1;         // [2]  GEMM 2 of the tile that used this feature buffer is complete
+  uint64_t* w_ready = d2_full + 1;         // [1]  W_k operand stored to tensor memory
   float* snorm = reinterpret_cast<float*>(bars + 32);        // [2][128]  -gamma log2e |k_t|^2, -inf if masked
-  float* ucomb = snorm + 2 * 128;                            // [2][128]
-  int* misc = reinterpret_cast<int*>(ucomb + 2 * 128);
+  float* ucomb = reinterpret_cast<float*>(ring);             // [kNG][128], written after the last MMA has read the ring
+  int* misc = reinterpret_cast<int*>(snorm + 2 * 128);
   volatile int* s_abort = misc;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 1);
 
@@ -97,6 +107,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
   float* S_out = p.S + (size_t)unit * D * R;
   float* u_out = p.u + (size_t)unit * R;
+  pdl_launch_next();                       // the reduction kernel may be scheduled; it waits for this grid's completion
   if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) *p.status = kStatusOk;
   if (n_mid == 0) {
     if (chunk == 0) {
@@ -112,146 +123,154 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   const int t1 = (int)((long long)n_tiles * (chunk + 1) / n_chunks);
   const int n_my = t1 - t0;                                   // >= 1
   const int row0 = (int)(cu_b + p.n_sink);                    // cache row of mid token 0
+  // Ring loads are issued in the order in which the tensor pipe consumes the tiles: K0, K1, V0, K2, V1, ...,
+  // V(last) (GEMM 1 of tile i+1 runs before GEMM 2 of tile i), so that no landed tile waits in a slot while a
+  // later one is consumed.  Sequence numbers of the key and the value tile of tile i:
+  auto seq_k = [&](int i) { return MODE == 2 ? 0 : (i == 0 ? 0 : 2 * i - 1); };
+  auto seq_v = [&](int i) { return MODE == 2 ? i : (2 * i + 2 < 2 * n_my - 1 ? 2 * i + 2 : 2 * n_my - 1); };
 
-  // ---- set-up: barriers, tensor memory, W_k operand tiles (scaled by log2 e, hi + lo)
+  // ---- set-up: barriers and tensor memory first, so that the producer can start the key/value
+  // stream while four warps (one per lane quadrant) store W_k (scaled by log2 e, hi + lo) to tensor memory
   if (tid == 0) {
-    for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 5); }
-    for (int s = 0; s < VS; ++s) { mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
+    for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&d1_full[s], 1); mbar_init(&p_ready[s], 8); mbar_init(&n_ready[s], 4);
+      mbar_init(&p_ready[s], kFWarps); mbar_init(&n_ready[s], 4); mbar_init(&d1_full[s], 1); mbar_init(&buf_free[s], 1);
     }
     mbar_init(d2_full, 1);
-    mbar_init(&g2_done[0], 1); mbar_init(&g2_done[1], 1);
+    mbar_init(w_ready, 4);
     mbar_fence_init();
     *s_abort = 0;
   }
   if (warp == 1) tmem_alloc(s_tmem, kBuildTmemCols);
-  if (MODE != 2) {
-    const float* W = p.w_k + (size_t)kvh * R * D;
-    constexpr int CPR = D / 8;
-    for (int i = tid; i < 128 * CPR; i += kBuildThreads) {
-      const int row = i / CPR, c = i % CPR;
-      unsigned hw[4] = {0, 0, 0, 0}, lw[4] = {0, 0, 0, 0};
-      if (row < R) {
-        const float4 w0 = *reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8);
-        const float4 w1 = *reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8 + 4);
-        const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float a0 = w[2 * e] * kLog2e, a1 = w[2 * e + 1] * kLog2e;
-          const __nv_bfloat16 h0 = __float2bfloat16_rn(a0), h1 = __float2bfloat16_rn(a1);
-          const __nv_bfloat16 l0 = __float2bfloat16_rn(a0 - __bfloat162float(h0));
-          const __nv_bfloat16 l1 = __float2bfloat16_rn(a1 - __bfloat162float(h1));
-          hw[e] = (unsigned)__bfloat16_as_ushort(h0) | ((unsigned)__bfloat16_as_ushort(h1) << 16);
-          lw[e] = (unsigned)__bfloat16_as_ushort(l0) | ((unsigned)__bfloat16_as_ushort(l1) << 16);
-        }
-      }
-      const uint32_t off = (c >> 3) * C::BOX + swz128(row, c & 7);
-      *reinterpret_cast<uint4*>(whi + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-      *reinterpret_cast<uint4*>(wlo + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-    }
-  }
-  fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
+  if (MODE != 2 && warp >= 2 && warp < 6) {
+    // thread = feature row j (tensor-memory lane); column c of the operand holds dims 2c, 2c + 1
+    const int j = (warp & 3) * 32 + lane;
+    const float* Wj = p.w_k + ((size_t)kvh * R + (j < R ? j : 0)) * D;
+#pragma unroll
+    for (int blk = 0; blk < D / 32; ++blk) {               // 32 dims -> 16 packed columns
+      uint32_t hw[16], lw[16];
+#pragma unroll
+      for (int f = 0; f < 8; ++f) {
+        float4 w4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j < R) w4 = __ldg(reinterpret_cast<const float4*>(Wj + blk * 32 + f * 4));
+        const float w[4] = {w4.x * kLog2e, w4.y * kLog2e, w4.z * kLog2e, w4.w * kLog2e};
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const __nv_bfloat162 hp = __floats2bfloat162_rn(w[2 * e], w[2 * e + 1]);      // .x (low half) = even dim
+          const __nv_bfloat162 lp =
+              __floats2bfloat162_rn(w[2 * e] - __bfloat162float(hp.x), w[2 * e + 1] - __bfloat162float(hp.y));
+          hw[2 * f + e] = *reinterpret_cast<const uint32_t*>(&hp);
+          lw[2 * f + e] = *reinterpret_cast<const uint32_t*>(&lp);
+        }
+      }
+      tmem_st_x16(tmem_addr(tmem_base, (warp & 3) * 32, kColW + blk * 16), hw);
+      tmem_st_x16(tmem_addr(tmem_base, (warp & 3) * 32, kColW + 64 + blk * 16), lw);
+    }
+    tc_wait_st();
+    tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(w_ready);
+  }
 
   if (warp == 0) {
     // ================================================================ TMA producer
     if (lane == 0) {
       bool ok = true;
-      const uint64_t pol = l2_policy_evict_first();        // K and V are read once
-      for (int it = 0; it < n_my && ok; ++it) {
-        const int row = row0 + (t0 + it) * kBT;
-        const int ks = it % KS, vs = it % VS;
-        if (MODE != 2) {
-          ok = mbar_wait(&k_empty[ks], ((uint32_t)(it / KS) & 1u) ^ 1u, s_abort);
-          if (!ok) break;
-          mbar_expect_tx(&k_full[ks], C::TILE);
+      int last_n[NS];                                      // last load issued into each slot
 #pragma unroll
-          for (int x = 0; x < BOXES; ++x)
-            tma_load_3d(kring + ks * C::TILE + x * C::BOX, &tmap_k, &k_full[ks], x * 64, row, kvh, pol);
-        }
-        ok = mbar_wait(&v_empty[vs], ((uint32_t)(it / VS) & 1u) ^ 1u, s_abort);
-        if (!ok && MODE == 2) break;
-        if (!ok) {
-          // the key copy just issued must land before shared memory is released
-          for (uint32_t w = 0; w < kWaitPolls; ++w) {
-            if (mbar_try_wait(&k_full[ks], (uint32_t)(it / KS) & 1u)) break;
-            __nanosleep(64);
-          }
-          break;
-        }
-        mbar_expect_tx(&v_full[vs], C::TILE);
+      for (int s = 0; s < NS; ++s) last_n[s] = -1;
+      const uint64_t pol = l2_policy_evict_first();        // K and V are read once
+      for (int n = 0; n < LPT * n_my && ok; ++n) {
+        const int slot = n % NS;
+        const bool is_key = MODE != 2 && n != 2 * n_my - 1 && (n == 0 || (n & 1) != 0);
+        const int it = MODE == 2 ? n : (n == 0 ? 0 : n == 2 * n_my - 1 ? n_my - 1 : is_key ? (n + 1) / 2 : n / 2 - 1);
+        const int row = row0 + (t0 + it) * kBT;
+        ok = mbar_wait(&empty[slot], ((uint32_t)(n / NS) & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+#pragma unroll
+        for (int s = 0; s < NS; ++s)
+          if (s == slot) last_n[s] = n;
+        mbar_expect_tx(&full[slot], C::TILE);
 #pragma unroll
         for (int x = 0; x < BOXES; ++x)
-          tma_load_3d(vring + vs * C::TILE + x * C::BOX, &tmap_v, &v_full[vs], x * 64, row, kvh, pol);
+          tma_load_3d(ring + slot * C::TILE + x * C::BOX, is_key ? &tmap_k : &tmap_v, &full[slot], x * 64, row, kvh, pol);
+      }
+      if (!ok) {
+        // every copy that was issued must land before shared memory is released
+#pragma unroll
+        for (int s = 0; s < NS; ++s)
+          for (uint32_t w = 0; last_n[s] >= 0 && w < kWaitPolls; ++w) {
+            if (mbar_try_wait(&full[s], (uint32_t)(last_n[s] / NS) & 1u)) break;
+            __nanosleep(64);
+          }
       }
     }
   } else if (warp == 1) {
-    // ================================================================ MMA issuer
-    if (lane == 0) {
+    // ================================================================ GEMM-1 issuer
+    if (MODE != 2 && lane == 0) {
       constexpr uint32_t idesc1 = umma_idesc_bf16(128, kBT, 0, 0);
-      constexpr uint32_t idesc2 = umma_idesc_bf16(128, D, 0, 1);
-      const uint64_t whi_d = umma_smem_desc(smem_u32(whi), 16, 1024);
-      const uint64_t wlo_d = umma_smem_desc(smem_u32(wlo), 16, 1024);
-      const uint64_t k_d = umma_smem_desc(smem_u32(kring), 16, 1024);
-      // value tile as an MN-major operand: 64-dim column blocks BOX bytes apart, groups of
-      // eight token rows 1024 bytes apart
-      const uint64_t v_d = umma_smem_desc(smem_u32(vring), C::BOX, 1024);
-      bool ok = true;
-      auto gemm2 = [&](int j) {
-        const int buf = j & 1, vs = j % VS;
-        ok = mbar_wait(&p_ready[buf], (uint32_t)(j >> 1) & 1u, s_abort) &&
-             mbar_wait(&v_full[vs], (uint32_t)(j / VS) & 1u, s_abort);
-        if (!ok) return;
-        tc_fence_after_sync();
-        const uint64_t vd = v_d + (uint64_t)((vs * C::TILE) >> 4);
-#pragma unroll
-        for (int kk = 0; kk < kBT / 16; ++kk) {
-          // tokens 16 kk .. 16 kk + 15: eight packed columns of Phi hi, then of Phi lo
-          const uint32_t hi_col = kColD1 + buf * 128 + (kk >> 2) * 64 + ((kk >> 1) & 1) * 16 + (kk & 1) * 8;
-          const uint32_t lo_col = kColLo + buf * 64 + (kk >> 2) * 32 + ((kk >> 1) & 1) * 16 + (kk & 1) * 8;
-          const uint64_t bd = vd + (uint64_t)((kk * 16 * 128) >> 4);
-          umma_ts(tmem_base + kColD2, tmem_base + hi_col, bd, idesc2, (j > 0 || kk > 0) ? 1u : 0u);
-          umma_ts(tmem_base + kColD2, tmem_base + lo_col, bd, idesc2, 1u);
-        }
-        tc_commit(&v_empty[vs]);
-        tc_commit(&g2_done[buf]);
-      };
-      if (MODE == 2) {
-        for (int it = 0; it + 1 < n_my && ok; ++it) gemm2(it);
-      }
-      for (int it = 0; MODE != 2 && it < n_my && ok; ++it) {
-        const int buf = it & 1, ks = it % KS;
-        // No wait for GEMM 2 of tile it-2, whose A operand lives where this accumulator goes:
-        // MMAs issued by one thread execute in issue order, and the feature warps touch the
-        // buffer only after d1_full of this tile.
-        ok = mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort);
+      const uint64_t ring_k = umma_smem_desc(smem_u32(ring), 16, 1024);
+      bool ok = mbar_wait(w_ready, 0, s_abort);
+      tc_fence_after_sync();
+      for (int it = 0; it < n_my && ok; ++it) {
+        const int buf = it & 1, nk = seq_k(it), ks = nk % NS;
+        // the buffer is free once GEMM 2 of tile it-2 has read its features
+        ok = mbar_wait(&full[ks], (uint32_t)(nk / NS) & 1u, s_abort) &&
+             (it < 2 || mbar_wait(&buf_free[buf], (uint32_t)((it - 2) >> 1) & 1u, s_abort));
         if (!ok) break;
         tc_fence_after_sync();
-        const uint64_t kd = k_d + (uint64_t)((ks * C::TILE) >> 4);
+        const uint64_t kd = ring_k + (uint64_t)((ks * C::TILE) >> 4);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-          const uint64_t wd = half == 0 ? whi_d : wlo_d;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint64_t off = (uint64_t)(((k >> 2) * C::BOX + (k & 3) * 32) >> 4);
-            umma_ss(tmem_base + kColD1 + buf * 128, wd + off, kd + off, idesc1, (half | k) ? 1u : 0u);
+            umma_ts(tmem_base + kColBuf + buf * 128, tmem_base + kColW + half * 64 + k * 8, kd + off, idesc1, (half | k) ? 1u : 0u);
           }
         }
         tc_commit(&d1_full[buf]);
-        tc_commit(&k_empty[ks]);
-        if (it > 0) gemm2(it - 1);
+        // the slot is released once GEMM 1 is complete and the norm warps have read the tile
+        ok = mbar_wait(&n_ready[buf], (uint32_t)(it >> 1) & 1u, s_abort);
+        if (!ok) break;
+        tc_commit(&empty[ks]);
       }
-      if (ok) gemm2(n_my - 1);
+    }
+  } else if (warp == kWarpG2) {
+    // ================================================================ GEMM-2 issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc2 = umma_idesc_bf16(128, D, 0, 1);
+      // value tile as an MN-major operand: 64-dim column blocks BOX bytes apart, groups of
+      // eight token rows 1024 bytes apart
+      const uint64_t ring_v = umma_smem_desc(smem_u32(ring), C::BOX, 1024);
+      bool ok = true;
+      for (int j = 0; j < n_my && ok; ++j) {
+        const int buf = j & 1, nv = seq_v(j), vs = nv % NS;
+        ok = mbar_wait(&p_ready[buf], (uint32_t)(j >> 1) & 1u, s_abort) &&
+             mbar_wait(&full[vs], (uint32_t)(nv / NS) & 1u, s_abort);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t vd = ring_v + (uint64_t)((vs * C::TILE) >> 4);
+#pragma unroll
+        for (int kk = 0; kk < kBT / 16; ++kk) {
+          // tokens 16 kk .. 16 kk + 15: eight packed columns of Phi hi, then of Phi lo, against sixteen rows of the value tile
+          const uint64_t bd = vd + (uint64_t)((kk * 16 * 128) >> 4);
+          const uint32_t a_col = kColBuf + buf * 128 + (kk * 16 / kTPT) * kTPT + (kk * 16 % kTPT) / 2;
+          umma_ts(tmem_base + kColD2, tmem_base + a_col, bd, idesc2, (j > 0 || kk > 0) ? 1u : 0u);
+          umma_ts(tmem_base + kColD2, tmem_base + a_col + kTPT / 2, bd, idesc2, 1u);
+        }
+        tc_commit(&empty[vs]);
+        tc_commit(&buf_free[buf]);
+      }
       if (ok) tc_commit(d2_full);
     }
-  } else if (warp < 10) {
+  } else if (warp < kWarpNorm) {
     // ================================================================ feature warps
     const int quad = warp & 3;                     // tensor-memory lane quadrant
-    const int h = (warp - 2) >> 2;                 // which 64 tokens of the tile
+    const int g = (warp - 2) >> 2;                 // which token group of the tile
     const int j = quad * 32 + lane;                // feature
     const float bj = (MODE != 2 && j < R) ? p.b_k[(size_t)kvh * R + j] * kLog2e : 0.f;
     float u_acc = 0.f;                             // sum of feature j over this thread's tokens
@@ -261,29 +280,33 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     for (int it = 0; it < n_my && ok; ++it) {
       const int buf = it & 1;
       const uint32_t ph = (uint32_t)(it >> 1) & 1u;
-      if (MODE == 2) {
-        // the feature buffer is free once GEMM 2 of tile it - 2 has read it; snorm says which tokens are in the mid-region
-        ok = mbar_wait(&n_ready[buf], ph, s_abort) && (it < 2 || mbar_wait(&g2_done[buf], ph ^ 1u, s_abort));
-      } else {
-        ok = mbar_wait(&d1_full[buf], ph, s_abort) && mbar_wait(&n_ready[buf], ph, s_abort);
-      }
+      // mode 2 has no GEMM 1 whose issuer would wait for the buffer
+      ok = (MODE == 2 ? (it < 2 || mbar_wait(&buf_free[buf], (uint32_t)((it - 2) >> 1) & 1u, s_abort))
+                      : mbar_wait(&d1_full[buf], ph, s_abort)) &&
+           mbar_wait(&n_ready[buf], ph, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      const float* sn = snorm + buf * 128 + h * 64;
+      const float* sn = snorm + buf * 128 + g * kTPT;
+      uint32_t hi[kTPT / 2], lo[kTPT / 2];         // this thread's tokens, packed in pairs
+      float vv[kTPT / 32][32];
+      if (MODE != 2) {
+        // this thread's whole accumulator slice into registers: the features go over the same columns
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        float v[32];
+        for (int c = 0; c < kTPT / 32; ++c)
+          tmem_ld_x32(tmem_addr(tmem_base, quad * 32, kColBuf + buf * 128 + g * kTPT + c * 32), vv[c]);
+        tc_wait_ld();
+      }
+#pragma unroll
+      for (int c = 0; c < kTPT / 32; ++c) {
+        float (&v)[32] = vv[c];
         if (MODE == 2) {
-          const int tok0 = (t0 + it) * kBT + h * 64 + c * 32;
+          // snorm says which tokens are in the mid-region
+          const int tok0 = (t0 + it) * kBT + g * kTPT + c * 32;
 #pragma unroll
           for (int e = 0; e < 32; ++e)
             v[e] = (cache_j != nullptr && sn[c * 32 + e] == 0.f) ? __ldcs(cache_j + (size_t)(tok0 + e) * R) : 0.f;
-        } else {
-          tmem_ld_x32(tmem_addr(tmem_base, quad * 32, kColD1 + buf * 128 + h * 64 + c * 32), v);
-          tc_wait_ld();
         }
-        uint32_t hi[16], lo[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           const float f0 = MODE == 2 ? v[2 * e] : ex2_approx(v[2 * e] + bj + sn[c * 32 + 2 * e]);
@@ -293,25 +316,28 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
           const __nv_bfloat162 hp = __floats2bfloat162_rn(f0, f1);          // .x (low half) = even token
           const __nv_bfloat162 lp =
               __floats2bfloat162_rn(f0 - __bfloat162float(hp.x), f1 - __bfloat162float(hp.y));
-          hi[e] = *reinterpret_cast<const uint32_t*>(&hp);
-          lo[e] = *reinterpret_cast<const uint32_t*>(&lp);
+          hi[c * 16 + e] = *reinterpret_cast<const uint32_t*>(&hp);
+          lo[c * 16 + e] = *reinterpret_cast<const uint32_t*>(&lp);
           if (MODE == 1 && cache_j) {
             // one token per store: the 32 lanes of the warp write 32 consecutive features
-            const int tok = (t0 + it) * kBT + h * 64 + c * 32 + 2 * e;
+            const int tok = (t0 + it) * kBT + g * kTPT + c * 32 + 2 * e;
             if (tok < n_mid) __stcs(cache_j + (size_t)tok * R, f0);
             if (tok + 1 < n_mid) __stcs(cache_j + (size_t)(tok + 1) * R, f1);
           }
         }
-        // hi goes over columns of this thread's own region that it has already read
-        tmem_st_x16(tmem_addr(tmem_base, quad * 32, kColD1 + buf * 128 + h * 64 + c * 16), hi);
-        tmem_st_x16(tmem_addr(tmem_base, quad * 32, kColLo + buf * 64 + h * 32 + c * 16), lo);
+      }
+      // over the columns this thread has read: packed columns hi (column c = tokens 2c, 2c + 1 of the group), then lo
+#pragma unroll
+      for (int c = 0; c < kTPT / 32; ++c) {
+        tmem_st_x16(tmem_addr(tmem_base, quad * 32, kColBuf + buf * 128 + g * kTPT + c * 16), *reinterpret_cast<const uint32_t(*)[16]>(&hi[c * 16]));
+        tmem_st_x16(tmem_addr(tmem_base, quad * 32, kColBuf + buf * 128 + g * kTPT + kTPT / 2 + c * 16), *reinterpret_cast<const uint32_t(*)[16]>(&lo[c * 16]));
       }
       tc_wait_st();
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&p_ready[buf]);
     }
-    // ---- S^T of this CTA's tiles -> partial (thread = feature, h = half of the dims)
+    // ---- S^T of this CTA's tiles -> partial (thread = feature; the first two token groups' warps take half of the dims each)
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(d2_full, 0, s_abort));
     if (ok) {
       tc_fence_after_sync();
@@ -319,29 +345,31 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
       constexpr int HALF = D / 2;
 #pragma unroll
       for (int c = 0; c < HALF / 32; ++c) {
-        float v[32];
-        tmem_ld_x32(tmem_addr(tmem_base, quad * 32, kColD2 + h * HALF + c * 32), v);
-        tc_wait_ld();
-        if (j < R) {
+        if (g < 2) {                                 // warp-uniform
+          float v[32];
+          tmem_ld_x32(tmem_addr(tmem_base, quad * 32, kColD2 + g * HALF + c * 32), v);
+          tc_wait_ld();
+          if (j < R) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) part[(size_t)(h * HALF + c * 32 + e) * R + j] = v[e];
+            for (int e = 0; e < 32; ++e) part[(size_t)(g * HALF + c * 32 + e) * R + j] = v[e];
+          }
         }
       }
-      ucomb[h * 128 + j] = u_acc;
+      ucomb[g * 128 + j] = u_acc;
     }
   } else {
     // ================================================================ key norms and masking
-    const int t = (warp - 10) * 32 + lane;         // token of the tile
+    const int t = (warp - kWarpNorm) * 32 + lane;  // token of the tile
     const float g2 = p.gamma_k * kLog2e;
     bool ok = true;
     for (int it = 0; it < n_my && ok; ++it) {
-      const int buf = it & 1, ks = it % KS;
+      const int buf = it & 1, nk = seq_k(it), ks = nk % NS;
       // snorm[buf] was last read by the feature warps for tile it-2: wait for their p_ready
-      ok = (MODE == 2 || mbar_wait(&k_full[ks], (uint32_t)(it / KS) & 1u, s_abort)) &&
+      ok = (MODE == 2 || mbar_wait(&full[ks], (uint32_t)(nk / NS) & 1u, s_abort)) &&
            mbar_wait(&p_ready[buf], ((uint32_t)(it >> 1) & 1u) ^ 1u, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      const unsigned char* tile = kring + ks * C::TILE;
+      const unsigned char* tile = ring + ks * C::TILE;
       float kn = 0.f;
 #pragma unroll
       for (int c = 0; MODE != 2 && c < D / 8; ++c) {
@@ -357,7 +385,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
       const bool valid = (t0 + it) * kBT + t < n_mid;
       snorm[buf * 128 + t] = valid ? -g2 * kn : -INFINITY;   // exp2(-inf) = 0 removes rows outside the mid-region
       __syncwarp();
-      if (lane == 0) { mbar_arrive(&n_ready[buf]); if (MODE != 2) mbar_arrive(&k_empty[ks]); }
+      if (lane == 0) mbar_arrive(&n_ready[buf]);             // the MMA issuer releases the key slot after this
     }
   }
 
@@ -373,12 +401,19 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     return;
   }
   float* part = p.partials + ((size_t)unit * p.chunks_per_unit + chunk) * ((size_t)D * R + R);
-  if (tid < R) part[(size_t)D * R + tid] = ucomb[tid] + ucomb[128 + tid];
+  if (tid < R) {
+    float us = 0.f;
+#pragma unroll
+    for (int g = 0; g < kNG; ++g) us += ucomb[g * 128 + tid];
+    part[(size_t)D * R + tid] = us;
+  }
 }
 
 // Adds the chunk partials of every unit in chunk order (fixed order: run-to-run identical).
+// Launched as a programmatic dependent of the build kernel: waits for that grid first.
 constexpr int kRedThreads = 256;
 __global__ void __launch_bounds__(kRedThreads) build_reduce_kernel(const BuildProblem p) {
+  pdl_wait();
   const int unit = blockIdx.y, b = unit / p.n_kv_heads;
   const int D = p.head_dim, R = p.n_feat, n_out = D * R + R;
   const long long len_b = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
@@ -417,8 +452,16 @@ static cudaError_t launch_build_t(const BuildProblem& p, const CUtensorMap& tk, 
   if (e != cudaSuccess) return e;
   // one output per thread: every thread's loads of all chunk partials are in flight at once
   const int n_out = p.head_dim * p.n_feat + p.n_feat;
-  build_reduce_kernel<<<dim3((n_out + kRedThreads - 1) / kRedThreads, p.n_kv_heads * p.batch), kRedThreads, 0, st>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((n_out + kRedThreads - 1) / kRedThreads, p.n_kv_heads * p.batch, 1);
+  cfg.blockDim = dim3(kRedThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, build_reduce_kernel, p);
 }
 
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tk, const CUtensorMap& tv, cudaStream_t st) {
