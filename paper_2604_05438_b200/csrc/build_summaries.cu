@@ -137,7 +137,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
       mbar_init(&p_ready[s], kFWarps); mbar_init(&n_ready[s], 4); mbar_init(&d1_full[s], 1); mbar_init(&buf_free[s], 1);
     }
     mbar_init(d2_full, 1);
-    mbar_init(w_ready, 4);
+    mbar_init(w_ready, 4 * (D / 32) <= kFWarps ? 4 * (D / 32) : 4);
     mbar_fence_init();
     *s_abort = 0;
   }
@@ -146,12 +146,14 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
-  if (MODE != 2 && warp >= 2 && warp < 6) {
+  // one warp per (lane quadrant, block of 32 dims) when there are enough feature warps, else one per quadrant
+  constexpr bool kSplitW = 4 * (D / 32) <= kFWarps;
+  if (MODE != 2 && warp >= 2 && warp < 2 + (kSplitW ? 4 * (D / 32) : 4)) {
     // thread = feature row j (tensor-memory lane); column c of the operand holds dims 2c, 2c + 1
     const int j = (warp & 3) * 32 + lane;
     const float* Wj = p.w_k + ((size_t)kvh * R + (j < R ? j : 0)) * D;
-#pragma unroll
-    for (int blk = 0; blk < D / 32; ++blk) {               // 32 dims -> 16 packed columns
+    const int blk0 = kSplitW ? (warp - 2) >> 2 : 0, blk1 = kSplitW ? blk0 + 1 : D / 32;
+    for (int blk = blk0; blk < blk1; ++blk) {              // 32 dims -> 16 packed columns
       uint32_t hw[16], lw[16];
 #pragma unroll
       for (int f = 0; f < 8; ++f) {
