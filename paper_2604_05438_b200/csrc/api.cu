@@ -134,9 +134,13 @@ void build_layout(const tkphi_kv_desc* kv, const Shape& sh, WsLayout* L) {
   size_t o = 0;
   L->status = o;        o += 256;
   L->zero_end = o;
-  // one CTA per SM over all units, never more chunks than 128-token tiles
+  // One CTA per SM over all units, and no chunk longer than 256 tiles of 128 tokens: long units are cut into
+  // more chunks than that (several CTAs per SM in turn), which balances the SMs when units x chunks does not
+  // divide by the SM count and bounds the length of a tensor-memory accumulation chain (every MMA rounds its
+  // fp32 accumulator once; over 2048 tiles the bias reached 6.5e-4 of max |S|).  Never more chunks than tiles.
   const int64_t max_tiles = sh.max_mid > 0 ? ((int64_t)sh.max_mid + 127) / 128 : 1;
   int64_t cpu = n_sm_cached() / sh.units;
+  if (cpu < (max_tiles + 255) / 256) cpu = (max_tiles + 255) / 256;
   if (cpu < 1) cpu = 1;
   if (cpu > max_tiles) cpu = max_tiles;
   L->chunks_per_unit = (int)cpu;
