@@ -86,6 +86,10 @@ enum {
  * Anchors (Eq. partition): the first n_sink and the last n_tail rows of each
  * sequence (their union when L_b < n_sink + n_tail); the mid-region is what lies
  * between, |M_b| = max(0, L_b - n_sink - n_tail).
+ * n_tail_seq_host / n_tail_seq_dev (optional; both NULL or both given, the same [batch]
+ * values >= 0 on the host and on the device) give every sequence a tail-anchor count of its
+ * own, which then replaces n_tail everywhere: sequences that have generated different
+ * numbers of tokens share a decode call this way (see tkphi_decode_step).
  */
 typedef struct {
   int32_t batch, n_q_heads, n_kv_heads, head_dim;
@@ -96,6 +100,8 @@ typedef struct {
   const void* k;                  /* device, bf16 */
   const void* v;                  /* device, bf16 */
   int64_t kv_stride_head, kv_stride_token; /* in elements */
+  const int32_t* n_tail_seq_host; /* host,   [batch] or NULL */
+  const int32_t* n_tail_seq_dev;  /* device, [batch] or NULL */
 } tkphi_kv_desc;
 
 /* phi(x) = exp(W x + b - gamma ||x||^2); row-major fp32 parameters on the device; w_q and
@@ -216,7 +222,8 @@ tkphi_status tkphi_topk_decode(const tkphi_kv_desc* kv, const void* q,
  * Generated tokens (Sec. 4.3, Eq. implemented_decode: tokens produced after the prefill
  * stay in the exact branch): append their rows to the cache and pass n_tail + n_gen as the
  * tail-anchor count of the decode call; the mid-region, and with it the meaning of (S, u)
- * built at prefill time with n_tail, is unchanged.  All sequences of a call share n_gen.
+ * built at prefill time with n_tail, is unchanged.  Sequences with different n_gen share a
+ * call through n_tail_seq (entry b = n_tail + n_gen_b).
  * Other arguments as for tkphi_topk_decode.
  */
 tkphi_status tkphi_decode_step(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, const void* q,

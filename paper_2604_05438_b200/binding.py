@@ -40,7 +40,7 @@ class _KvDesc(C.Structure):
                 ("head_dim", C.c_int32), ("n_feat", C.c_int32), ("n_sink", C.c_int32),
                 ("n_tail", C.c_int32), ("cu_seqlens_host", C.c_void_p), ("cu_seqlens_dev", C.c_void_p),
                 ("k", C.c_void_p), ("v", C.c_void_p), ("kv_stride_head", C.c_int64),
-                ("kv_stride_token", C.c_int64)]
+                ("kv_stride_token", C.c_int64), ("n_tail_seq_host", C.c_void_p), ("n_tail_seq_dev", C.c_void_p)]
 
 
 class _PhiDesc(C.Structure):
@@ -140,11 +140,18 @@ class KVCache:
     n_sink: int
     n_tail: int
     cu_seqlens_dev: Optional[torch.Tensor] = None
+    n_tail_seq: Optional[np.ndarray] = None        # int32 [batch]: per-sequence tail-anchor counts (replace n_tail)
+    n_tail_seq_dev: Optional[torch.Tensor] = None
 
     def __post_init__(self):
         self.cu_seqlens = np.ascontiguousarray(self.cu_seqlens, dtype=np.int64)
         if self.cu_seqlens_dev is None:
             self.cu_seqlens_dev = torch.from_numpy(self.cu_seqlens).to(self.k.device)
+        if self.n_tail_seq is not None:
+            self.n_tail_seq = np.ascontiguousarray(self.n_tail_seq, dtype=np.int32)
+            assert self.n_tail_seq.shape == (len(self.cu_seqlens) - 1,)
+            if self.n_tail_seq_dev is None:
+                self.n_tail_seq_dev = torch.from_numpy(self.n_tail_seq).to(self.k.device)
 
     @property
     def batch(self) -> int:
@@ -156,7 +163,9 @@ class KVCache:
         assert k.stride() == v.stride() and k.stride(2) == 1
         return _KvDesc(self.batch, self.n_q_heads, k.shape[0], k.shape[2], self.n_feat, self.n_sink,
                        self.n_tail, self.cu_seqlens.ctypes.data, self.cu_seqlens_dev.data_ptr(),
-                       k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1))
+                       k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1),
+                       None if self.n_tail_seq is None else self.n_tail_seq.ctypes.data,
+                       None if self.n_tail_seq is None else self.n_tail_seq_dev.data_ptr())
 
 
 @dataclass

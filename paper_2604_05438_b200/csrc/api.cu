@@ -30,6 +30,11 @@ struct Shape {
   long long score_tiles;          // tiles of the scoring kernel (all units)
 };
 
+// Tail-anchor count of sequence b: the per-sequence array when given, else n_tail.
+inline int64_t tail_host(const tkphi_kv_desc* kv, int b) {
+  return kv->n_tail_seq_host ? kv->n_tail_seq_host[b] : kv->n_tail;
+}
+
 tkphi_status validate_kv(const tkphi_kv_desc* kv, Shape* sh, bool need_data) {
   if (!kv) return fail(TKPHI_ERR_INVALID_ARG, "kv descriptor is NULL");
   if (kv->batch < 1 || kv->batch > kMaxBatch)
@@ -44,6 +49,11 @@ tkphi_status validate_kv(const tkphi_kv_desc* kv, Shape* sh, bool need_data) {
   if (kv->n_q_heads / kv->n_kv_heads > 8)
     return fail(TKPHI_ERR_UNSUPPORTED, "group size %d > 8", kv->n_q_heads / kv->n_kv_heads);
   if (kv->n_sink < 0 || kv->n_tail < 0) return fail(TKPHI_ERR_INVALID_ARG, "negative anchor count");
+  if ((kv->n_tail_seq_host == nullptr) != (kv->n_tail_seq_dev == nullptr))
+    return fail(TKPHI_ERR_INVALID_ARG, "n_tail_seq_host and n_tail_seq_dev must both be NULL or both be given");
+  if (kv->n_tail_seq_host)
+    for (int b = 0; b < kv->batch; ++b)
+      if (kv->n_tail_seq_host[b] < 0) return fail(TKPHI_ERR_INVALID_ARG, "n_tail_seq[%d] = %d is negative", b, kv->n_tail_seq_host[b]);
   if (!kv->cu_seqlens_host) return fail(TKPHI_ERR_INVALID_ARG, "cu_seqlens_host is NULL");
   const int64_t* cu = kv->cu_seqlens_host;
   if (cu[0] != 0) return fail(TKPHI_ERR_INVALID_ARG, "cu_seqlens[0] must be 0");
@@ -53,7 +63,7 @@ tkphi_status validate_kv(const tkphi_kv_desc* kv, Shape* sh, bool need_data) {
     if (len < 1) return fail(TKPHI_ERR_INVALID_ARG, "sequence %d has length %lld (< 1)", b, (long long)len);
     if (cu[b + 1] >= (1ll << 31)) return fail(TKPHI_ERR_INVALID_ARG, "more than 2^31-1 cache rows");
     if (len > sh->max_len) sh->max_len = (int)len;
-    const int64_t mid = len - kv->n_sink - kv->n_tail;
+    const int64_t mid = len - kv->n_sink - tail_host(kv, b);
     if (mid > sh->max_mid) sh->max_mid = (int)mid;
   }
   sh->total_tokens = cu[kv->batch];
@@ -93,13 +103,13 @@ tkphi_status validate_topk(const tkphi_kv_desc* kv, const int32_t* topk_host, in
   sh->score_tiles = 0;
   for (int b = 0; b < kv->batch; ++b) {
     const int64_t len = cu[b + 1] - cu[b];
-    int64_t mid = len - kv->n_sink - kv->n_tail;
+    int64_t mid = len - kv->n_sink - tail_host(kv, b);
     if (mid < 0) mid = 0;
     if (topk_host[b] < 0 || topk_host[b] > mid)
       return fail(TKPHI_ERR_INVALID_ARG, "topk[%d] = %d outside [0, |M| = %lld]", b, topk_host[b], (long long)mid);
     if (topk_host[b] > topk_max)
       return fail(TKPHI_ERR_INVALID_ARG, "topk[%d] = %d exceeds topk_max = %d", b, topk_host[b], topk_max);
-    if (!allow_empty_support && topk_host[b] == 0 && kv->n_sink == 0 && kv->n_tail == 0)
+    if (!allow_empty_support && topk_host[b] == 0 && kv->n_sink == 0 && tail_host(kv, b) == 0)
       return fail(TKPHI_ERR_INVALID_ARG, "sequence %d has an empty exact support (no anchors, topk = 0)", b);
     if (topk_host[b] > 0) sh->score_tiles += (int64_t)kv->n_kv_heads * ((mid + tk - 1) / tk);
     if (mid > 2097152)
@@ -120,7 +130,13 @@ void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, W
   L->wk_img = o;        o = align_up(o + (size_t)kv->n_kv_heads * 2 * kv->n_feat * kv->head_dim * 2, 1024);
   L->idx = o;           o = align_up(o + sizeof(int) * (size_t)sh.rows * (topk_max > 0 ? topk_max : 1), 256);
   L->aq = o;            o = align_up(o + sizeof(float) * (size_t)sh.rows * aq_stride(kv->n_feat, kv->head_dim), 256);
-  int64_t max_support = (int64_t)kv->n_sink + kv->n_tail + topk_max;
+  int64_t max_tail = kv->n_tail;
+  if (kv->n_tail_seq_host) {
+    max_tail = 0;
+    for (int b = 0; b < kv->batch; ++b)
+      if (kv->n_tail_seq_host[b] > max_tail) max_tail = kv->n_tail_seq_host[b];
+  }
+  int64_t max_support = (int64_t)kv->n_sink + max_tail + topk_max;
   if (max_support > sh.max_len) max_support = sh.max_len;
   L->max_slices = (int)((max_support + kSlice - 1) / kSlice);
   if (L->max_slices < 1) L->max_slices = 1;
@@ -342,6 +358,7 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   Problem p{};
   p.batch = kv->batch; p.n_q_heads = kv->n_q_heads; p.n_kv_heads = kv->n_kv_heads;
   p.head_dim = kv->head_dim; p.n_feat = kv->n_feat; p.n_sink = kv->n_sink; p.n_tail = kv->n_tail;
+  p.n_tail_seq = kv->n_tail_seq_dev;
   p.group = kv->n_q_heads / kv->n_kv_heads;
   p.cu_seqlens = reinterpret_cast<const long long*>(kv->cu_seqlens_dev);
   p.topk = topk_dev; p.topk_max = topk_max > 0 ? topk_max : 1;
@@ -412,7 +429,7 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
     for (int b = 0; b < kv->batch; ++b) {
       const long long len_b = kv->cu_seqlens_host[b + 1] - kv->cu_seqlens_host[b];
       const long long n_a1 = len_b < kv->n_sink ? len_b : kv->n_sink;
-      long long ts = len_b - kv->n_tail;
+      long long ts = len_b - tail_host(kv, b);
       if (ts < kv->n_sink) ts = kv->n_sink;
       if (ts > len_b) ts = len_b;
       const long long n_e = n_a1 + topk_host[b] + (len_b - ts);
@@ -447,7 +464,7 @@ tkphi_status build_common(const tkphi_kv_desc* kv, const float* w_k, const float
   char* w = static_cast<char*>(workspace);
   BuildProblem p{};
   p.batch = kv->batch; p.n_kv_heads = kv->n_kv_heads; p.head_dim = kv->head_dim; p.n_feat = kv->n_feat;
-  p.n_sink = kv->n_sink; p.n_tail = kv->n_tail;
+  p.n_sink = kv->n_sink; p.n_tail = kv->n_tail; p.n_tail_seq = kv->n_tail_seq_dev;
   p.cu_seqlens = reinterpret_cast<const long long*>(kv->cu_seqlens_dev);
   p.k = static_cast<const __nv_bfloat16*>(kv->k); p.v = static_cast<const __nv_bfloat16*>(kv->v);
   p.stride_head = kv->kv_stride_head; p.stride_token = kv->kv_stride_token;

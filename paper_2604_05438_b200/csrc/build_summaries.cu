@@ -104,7 +104,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   const int R = p.n_feat;
   const int unit = b * p.n_kv_heads + kvh;
   const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
-  const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
+  const int n_mid = mid_len(len_b, p.n_sink, tail_of(p, b));
   float* S_out = p.S + (size_t)unit * D * R;
   float* u_out = p.u + (size_t)unit * R;
   pdl_launch_next();                       // the reduction kernel may be scheduled; it waits for this grid's completion
@@ -419,7 +419,7 @@ __global__ void __launch_bounds__(kRedThreads) build_reduce_kernel(const BuildPr
   const int unit = blockIdx.y, b = unit / p.n_kv_heads;
   const int D = p.head_dim, R = p.n_feat, n_out = D * R + R;
   const long long len_b = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
-  const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
+  const int n_mid = mid_len(len_b, p.n_sink, tail_of(p, b));
   if (n_mid == 0) return;                              // the build kernel wrote zeros
   const int n_tiles = (n_mid + kBT - 1) / kBT;
   const int n_chunks = n_tiles < p.chunks_per_unit ? n_tiles : p.chunks_per_unit;

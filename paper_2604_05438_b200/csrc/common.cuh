@@ -34,6 +34,7 @@ struct MlpParams {
 // Everything the kernels need to know about one layer call.
 struct Problem {
   int batch, n_q_heads, n_kv_heads, head_dim, n_feat, n_sink, n_tail, group;
+  const int* n_tail_seq;           // device [batch] per-sequence tail-anchor counts, or null: n_tail for all
   const long long* cu_seqlens;     // device [batch+1]
   const int* topk;                 // device [batch] (null for the build)
   int topk_max;
@@ -74,6 +75,7 @@ struct Problem {
 
 struct BuildProblem {
   int batch, n_kv_heads, head_dim, n_feat, n_sink, n_tail;
+  const int* n_tail_seq;           // as in Problem
   const long long* cu_seqlens;
   const __nv_bfloat16* k;
   const __nv_bfloat16* v;
@@ -107,6 +109,11 @@ __host__ __device__ inline int score_tile_keys(int head_dim) { return head_dim =
 __device__ __forceinline__ int mid_len(long long n, int n_sink, int n_tail) {
   long long m = n - n_sink - n_tail;
   return m > 0 ? (int)m : 0;
+}
+// Tail-anchor count of sequence b (P: Problem or BuildProblem).
+template <typename P>
+__device__ __forceinline__ int tail_of(const P& p, int b) {
+  return p.n_tail_seq ? __ldg(p.n_tail_seq + b) : p.n_tail;
 }
 
 // Order-preserving map from fp32 to uint32: larger float <=> larger key.

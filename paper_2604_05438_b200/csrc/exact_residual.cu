@@ -297,7 +297,7 @@ __global__ void __launch_bounds__(kExThreads) exact_residual_kernel(const Proble
   const int K = p.topk[b];
   const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
   const int nA1 = (int)(len_b < p.n_sink ? len_b : p.n_sink);
-  long long ts = len_b - p.n_tail;
+  long long ts = len_b - tail_of(p, b);
   if (ts < p.n_sink) ts = p.n_sink;
   if (ts > len_b) ts = len_b;
   const int tail_start = (int)ts, n_tail_eff = (int)(len_b - ts);
@@ -543,7 +543,7 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
   auto pairs_of = [&](int b) {
     const long long len_b = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
     const int nA1 = (int)(len_b < p.n_sink ? len_b : p.n_sink);
-    long long ts = len_b - p.n_tail;
+    long long ts = len_b - tail_of(p, b);
     if (ts < p.n_sink) ts = p.n_sink;
     if (ts > len_b) ts = len_b;
     const int nE = nA1 + p.topk[b] + (int)(len_b - ts);
@@ -600,7 +600,7 @@ exact_residual_stream_kernel(const __grid_constant__ CUtensorMap gmap_k, const _
     it.len_b = p.cu_seqlens[lo + 1] - it.cu_b;
     it.K = p.topk[lo];
     it.nA1 = (int)(it.len_b < p.n_sink ? it.len_b : p.n_sink);
-    long long ts = it.len_b - p.n_tail;
+    long long ts = it.len_b - tail_of(p, lo);
     if (ts < p.n_sink) ts = p.n_sink;
     if (ts > it.len_b) ts = it.len_b;
     it.tail_start = (int)ts;

@@ -102,7 +102,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
     for (int i = 0; i < per; ++i) {
       int b = b0 + i;
       if (b < batch) {
-        int nm = mid_len(p.cu_seqlens[b + 1] - p.cu_seqlens[b], p.n_sink, p.n_tail);
+        int nm = mid_len(p.cu_seqlens[b + 1] - p.cu_seqlens[b], p.n_sink, tail_of(p, b));
         int nt = (p.topk[b] > 0) ? (nm + TK - 1) / TK : 0;
         local += nt * n_kv;
       }
@@ -114,7 +114,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
       int b = b0 + i;
       if (b < batch) {
         pre[b] = run;
-        int nm = mid_len(p.cu_seqlens[b + 1] - p.cu_seqlens[b], p.n_sink, p.n_tail);
+        int nm = mid_len(p.cu_seqlens[b + 1] - p.cu_seqlens[b], p.n_sink, tail_of(p, b));
         int nt = (p.topk[b] > 0) ? (nm + TK - 1) / TK : 0;
         run += nt * n_kv;
       }
@@ -255,7 +255,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_k, const Problem p) {
           cur_b = cc.b; cur_kvh = cc.kvh;
           const long long cu_b = p.cu_seqlens[cur_b];
           len_b = p.cu_seqlens[cur_b + 1] - cu_b;
-          n_mid = mid_len(len_b, p.n_sink, p.n_tail);
+          n_mid = mid_len(len_b, p.n_sink, tail_of(p, cur_b));
           my_row = p.scores + score_row_base(p, cur_b, cur_kvh * G, cu_b, len_b) + (long long)g * len_b;
         }
         // the other read-back warp's tile (every accumulator buffer belongs to one warp: their number is even)

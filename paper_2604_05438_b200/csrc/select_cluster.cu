@@ -116,7 +116,7 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
   const int row = blockIdx.y, b = row / p.n_q_heads, hq = row % p.n_q_heads;
   const int K = p.topk[b];
   const long long cu_b = p.cu_seqlens[b], len_b = p.cu_seqlens[b + 1] - cu_b;
-  const int n_mid = mid_len(len_b, p.n_sink, p.n_tail);
+  const int n_mid = mid_len(len_b, p.n_sink, tail_of(p, b));
   const float* srow = p.scores + score_row_base(p, b, hq, cu_b, len_b);
   const int n_chunks = (n_mid + kSelChunk - 1) / kSelChunk;
   const int rounds = (n_chunks + csize - 1) / csize;       // per CTA

@@ -78,6 +78,18 @@ def test_invalid_arguments_are_rejected_before_any_launch(lib):
     assert _decode(lib, dd, [1]) == -1
     dd, _c = _desc([0, 100], n_sink=0, n_tail=0)
     assert _decode(lib, dd, [0]) == -1 and b"empty exact support" in lib.tkphi_last_error()
+    # per-sequence tail counts: both pointers or neither, no negative entry; they replace n_tail in every bound
+    tails = np.array([8, 90], np.int32)
+    dd, _c = _desc([0, 100, 300])
+    dd.n_tail_seq_host = tails.ctypes.data
+    assert _decode(lib, dd, [5, 6]) == -1 and b"n_tail_seq" in lib.tkphi_last_error()
+    dd.n_tail_seq_dev = 0x7000
+    assert _decode(lib, dd, [5, 6], ws=0) == -3
+    assert _decode(lib, dd, [89, 6]) == -1 and b"topk[0]" in lib.tkphi_last_error()      # |M_0| = 100 - 4 - 8 = 88
+    assert _decode(lib, dd, [88, 107]) == -1 and b"topk[1]" in lib.tkphi_last_error()    # |M_1| = 200 - 4 - 90 = 106
+    assert _decode(lib, dd, [88, 106], ws=0) == -3
+    tails[1] = -1
+    assert _decode(lib, dd, [5, 6]) == -1
     assert lib.tkphi_topk_decode(None, 0x4000, None, None, 0, None, 0x5000, 0x10000, 1 << 30, None) == -1
 
 

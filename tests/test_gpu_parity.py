@@ -324,6 +324,60 @@ def test_generated_tokens_stay_exact():
         assert PU.max_rel(out["y"][0, hq], y0) <= PU.Y_TOL, hq
 
 
+def test_sequences_with_different_tail_counts_share_a_call():
+    """Per-sequence tail-anchor counts (n_tail_seq): the build takes a different n_tail per sequence, and
+    the decode call n_tail_b + n_gen_b over caches that have grown by different numbers of generated tokens."""
+    import paper_2604_05438_b200 as T
+    cfg = _cfg("c1_1b_4k", n_q_heads=8, n_kv_heads=2)
+    dev = torch.device("cuda:0")
+    L = [1500, 700, 300]
+    tails = np.array([16, 40, 3], np.int32)
+    n_gen = np.array([37, 0, 5], np.int32)
+    inp = make_layer_inputs(cfg, 17, seq_lens=[l + int(g) for l, g in zip(L, n_gen)], n_steps=1)
+    phi = make_phi_params(cfg, 17, kind="visible", bk_shift=torch.full((cfg.n_kv_heads,), 2.0))
+    # prefill cache: the first L_b rows of every sequence
+    rows = np.concatenate([np.arange(int(inp.cu_seqlens[b]), int(inp.cu_seqlens[b]) + L[b]) for b in range(3)])
+    cu_pre = np.concatenate([[0], np.cumsum(L)]).astype(np.int64)
+    kp, vp = inp.k[:, rows].contiguous().to(dev), inp.v[:, rows].contiguous().to(dev)
+    kv_pre = T.KVCache(kp, vp, cu_pre, cfg.n_q_heads, cfg.n_feat, cfg.n_sink, 999, n_tail_seq=tails)   # n_tail itself is ignored
+    pd = phi.to(dev)
+    maps = T.PhiMaps(pd.w_q, pd.b_q, pd.w_k, pd.b_k, pd.gamma_q, pd.gamma_k)
+    B, Hq, Hkv, d, r = 3, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_feat
+    S = torch.full((B, Hkv, d, r), float("nan"), device=dev)
+    u = torch.full((B, Hkv, r), float("nan"), device=dev)
+    wsb = torch.empty(T.workspace_bytes(kv_pre, None, 0, T.WS_BUILD), dtype=torch.uint8, device=dev)
+    T.build_summaries(kv_pre, maps, S, u, wsb)
+    # decode over the grown caches
+    kv = T.KVCache(inp.k.to(dev), inp.v.to(dev), inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, cfg.n_sink, 0,
+                   n_tail_seq=tails + n_gen)
+    topk = np.array([29, 13, 6], np.int32)
+    tmax = int(topk.max())
+    ws = torch.empty(T.workspace_bytes(kv, topk, tmax, T.WS_DECODE_STEP), dtype=torch.uint8, device=dev)
+    idx = torch.full((B, Hq, tmax), -7, dtype=torch.int32, device=dev)
+    y = torch.full((B, Hq, d), float("nan"), device=dev)
+    T.decode_step(kv, maps, inp.q[0].to(dev).contiguous(), topk, torch.from_numpy(topk).to(dev), tmax, S, u, idx, y,
+                  None, 0, ws)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 0 and T.device_status(wsb) == 0
+    Sh, uh, yh, ih = S.cpu().double().numpy(), u.cpu().double().numpy(), y.cpu().numpy(), idx.cpu().numpy()
+    for b in range(B):
+        for kvh in range(Hkv):
+            K, V = PU.seq_arrays(inp, b, kvh)
+            S0, u0 = O.build_summaries(K[:L[b]], V[:L[b]], phi.w_k[kvh].double().numpy(), phi.b_k[kvh].double().numpy(),
+                                       phi.gamma_k, cfg.n_sink, int(tails[b]))
+            assert PU.note("S_rel_err", PU.max_rel(Sh[b, kvh], S0)) <= PU.SU_TOL, (b, kvh)
+            assert PU.note("u_rel_err", PU.max_rel(uh[b, kvh], u0)) <= PU.SU_TOL, (b, kvh)
+        for hq in range(Hq):
+            kvh = hq // cfg.group
+            K, V = PU.seq_arrays(inp, b, kvh)
+            q64 = inp.q[0, b, hq].double().numpy()
+            kk = int(topk[b])
+            ret = PU.check_selection(q64, K[:L[b]], cfg.n_sink, int(tails[b]), kk, ih[b, hq])
+            y0, _ = O.topkphi_attention_generated(q64, K, V, L[b], cfg.n_sink, int(tails[b]), kk, *_phi_arrays(phi, hq, kvh),
+                                                  S=Sh[b, kvh], u=uh[b, kvh], retrieved=ret)
+            assert PU.note("y_rel_err", PU.max_rel(yh[b, hq], y0)) <= PU.Y_TOL, (b, hq)
+
+
 def test_results_are_run_to_run_identical():
     cfg = CONFIGS["c1_1b_4k"]
     inp = make_layer_inputs(cfg, 12, seq_lens=[2500], n_steps=1)
