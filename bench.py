@@ -280,7 +280,7 @@ def run_ours(args, rank, world, device):
         "hbm_frac_of_measured_peak": ab["total"] / (ms * 1e-3) / 1e9 / peak,
         "algorithmic_bytes_per_step": ab["total"],
         "steps_per_s_all_gpus": whole_job_steps_per_s(ms, world),
-        "gpu_launches": args.steps * n_layers * (4 if (args.phi_cache or args.mlp_phi) else 3),
+        "gpu_launches": args.steps * n_layers * (8 if args.mlp_phi else 4 if args.phi_cache else 3),
         "e2e": {"value": e2e_ms * 1e3, "unit": "us/step", "h2d_bytes_per_step": q_stage.numel() * 2,
                 "d2h_bytes_per_step": y_host.numel() * 4},
         "build": build_info(build_ms, n_layers, Hkv, sum(max(0, n - cfg.n_sink - cfg.n_tail) for n in seq_lens), d, r,

@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtkphi.so")
 SOURCES = ["api.cu", "score.cu", "select_cluster.cu", "exact_residual.cu", "build_summaries.cu", "static_scratch.cu",
            "selftest.cu", "cached_features.cu",
-           "mlp_features.cu"]
+           "mlp_features.cu", "mlp_query.cu"]
 HEADERS = ["common.cuh", "sm100.cuh", "feature_jobs.cuh", os.path.join("..", "..", "include", "tkphi.h")]
 
 

@@ -143,6 +143,8 @@ void decode_layout(const tkphi_kv_desc* kv, const Shape& sh, int32_t topk_max, W
   L->partial_stride = 4 + 2 * kv->head_dim;
   L->partials = o;      o = align_up(o + sizeof(float) * (size_t)sh.rows * L->max_slices * L->partial_stride, 256);
   L->zbuf = o;          o = align_up(o + sizeof(float) * (size_t)sh.rows * (topk_max > 0 ? topk_max : 1), 256);
+  // layer outputs of the query-side MLP feature map at its largest hidden width (three vectors and the exponents per row)
+  L->mlp_vec = o;       o = align_up(o + sizeof(float) * (size_t)sh.rows * (3 * 512 + kv->n_feat), 256);
   L->total = o;
 }
 
@@ -367,6 +369,7 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
   p.q = static_cast<const __nv_bfloat16*>(q);
   if (with_phi && mlp_q) {
     p.mlp_q = mlp_params(mlp_q);
+    p.mlp_vec = reinterpret_cast<float*>(w + L.mlp_vec);
     p.S = S; p.u = u;
     if (!(flags & TKPHI_FLAG_NOSUB)) {
       p.phi_cache = mlp_cache;
@@ -396,6 +399,11 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
 
   p.zero_bytes = L.zero_end;
   cudaError_t e;
+  if (p.mlp_q.w_s) {      // the four layers of the query-side MLP, before the key stream
+    ScopedSpan sp(cs, TKPHI_KERNEL_MLP);
+    e = launch_mlp_query(p, cs);
+    if (e != cudaSuccess) return cuda_fail(e, "query-side MLP launch");
+  }
   // The scoring kernel also clears the workspace counters; without keys to score a plain
   // memset does.  The selection kernel carries the query-side feature work on extra clusters.
   if (sh.score_tiles > 0) {

@@ -46,6 +46,7 @@ struct Problem {
   const float* w_q; const float* b_q; const float* w_k; const float* b_k;
   float gamma_q, gamma_k;
   MlpParams mlp_q;                 // query-side MLP maps (mlp_q.w_s != nullptr: used instead of w_q, b_q, gamma_q)
+  float* mlp_vec;                  // their per-row layer outputs: [rows][g0 (E) | h (E) | g1 (E) | log phi_q (r)]
   // cached key features (optional): phi_k rows [n_kv_heads][total_tokens][n_feat], and where the
   // decode step keeps z_i = <phi_q, phi_k(k_i)> / exp(m_q) of the retrieved tokens: [rows][topk_max]
   const float* phi_cache; long long total_tokens;
@@ -93,7 +94,7 @@ struct BuildProblem {
 // Host-side byte offsets of the workspace pieces.
 struct WsLayout {
   size_t status, row_counter, zero_end;
-  size_t scores, wk_img, idx, aq, partials, zbuf, total;
+  size_t scores, wk_img, idx, aq, partials, zbuf, mlp_vec, total;
   int max_slices, partial_stride;
   // build
   size_t b_partials; int chunks_per_unit;
@@ -208,6 +209,7 @@ cudaError_t launch_select(const Problem& p, int max_mid, int n_sm, cudaStream_t 
 cudaError_t launch_exact_residual(const Problem& p, const CUtensorMap& gk, const CUtensorMap& gv, long long n_pairs, int n_sm,
                                   cudaStream_t stream);
 cudaError_t launch_cached_z(const Problem& p, cudaStream_t stream);
+cudaError_t launch_mlp_query(const Problem& p, cudaStream_t stream);
 
 // One dense layer of the MLP feature map on the tensor cores (mlp_features.cu):
 // out[h][m][n] = epilogue(sum_k A[h][m][k] W[h][n][k] + bias[h][n]).

@@ -14,55 +14,10 @@ namespace tkphi {
 // unsubtracted residual terms S_M w (d values) and w . u_M.  Row layout of p.aq:
 // [0, r) w, [r] m_q, [r+1] w . u_M, [r+4, r+4+d) S_M w, [r+4+d, 2r+4+d) log2 w.
 
-// y[i] = f(i, sum_c W[i][c] x[c]) for i < n_rows: warp w takes rows w, w + NT/32, ...; its lanes read a
-// row coalesced (n_cols a multiple of 4, x in shared memory) and add up in a fixed order.
-template <int NT, typename F>
-__device__ __forceinline__ void matvec_rows(const float* W, int n_rows, int n_cols, const float* x, F&& f) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int i = warp; i < n_rows; i += NT / 32) {
-    const float* wr = W + (size_t)i * n_cols;
-    float acc = 0.f;
-    for (int c = 4 * lane; c < n_cols; c += 128) {
-      const float4 w4 = __ldg(reinterpret_cast<const float4*>(wr + c));
-      acc = fmaf(w4.x, x[c], fmaf(w4.y, x[c + 1], fmaf(w4.z, x[c + 2], fmaf(w4.w, x[c + 3], acc))));
-    }
-    acc = warp_sum(acc);
-    if (lane == 0) f(i, acc);
-  }
-}
-
-// log phi_q(q) of the paper's ReZero-MLP feature map (App. C.2) for one query head, by all NT threads
-// of a CTA: g0 = W_s x + b_s; Delta = W_2 GeLU(W_1 g0 + b_1) + b_2; g1 = g0 + alpha Delta; a = W_o g1 + b_o.
-// x: the query in shared memory; scratch: 3 d_emb floats of shared memory; a_out: n_feat floats of shared memory.
+// Stage 1, by all NT threads of a CTA: w and m_q of query row `row`.  With the MLP feature map on the
+// query side the exponents log phi_q(q) come from the layer kernels that ran before (mlp_query.cu).
 template <int NT>
-__device__ void mlp_phi_q_log(const Problem& p, int hq, const float* x, float* scratch, float* a_out) {
-  const MlpParams& m = p.mlp_q;
-  const int E = m.d_emb, D = p.head_dim, r = p.n_feat;
-  float* g0 = scratch;
-  float* hbuf = scratch + E;
-  float* g1 = scratch + 2 * E;
-  const float* bs = m.b_s + (size_t)hq * E;
-  matvec_rows<NT>(m.w_s + (size_t)hq * E * D, E, D, x, [&](int i, float acc) { g0[i] = acc + bs[i]; });
-  __syncthreads();
-  const float* b1 = m.b_1 + (size_t)hq * E;
-  matvec_rows<NT>(m.w_1 + (size_t)hq * E * E, E, E, g0, [&](int i, float acc) {
-    const float t = acc + b1[i];
-    hbuf[i] = 0.5f * t * (1.f + erff(t * 0.70710678118654752f));
-  });
-  __syncthreads();
-  const float* b2 = m.b_2 + (size_t)hq * E;
-  const float al = m.alpha[hq];
-  matvec_rows<NT>(m.w_2 + (size_t)hq * E * E, E, E, hbuf, [&](int i, float acc) { g1[i] = fmaf(al, acc + b2[i], g0[i]); });
-  __syncthreads();
-  const float* bo = m.b_o + (size_t)hq * r;
-  matvec_rows<NT>(m.w_o + (size_t)hq * r * E, r, E, g1, [&](int i, float acc) { a_out[i] = acc + bo[i]; });
-  __syncthreads();
-}
-
-// Stage 1, by all NT threads of a CTA: w and m_q of query row `row`.  mlp_scratch: 3 d_emb floats of
-// shared memory, used when the query side is the MLP feature map.
-template <int NT>
-__device__ void phi_q_stage1(const Problem& p, int row, float* mlp_scratch) {
+__device__ void phi_q_stage1(const Problem& p, int row) {
   __shared__ float s_q[128];
   __shared__ float s_a[128];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -73,8 +28,9 @@ __device__ void phi_q_stage1(const Problem& p, int row, float* mlp_scratch) {
   const float* W = p.w_q + (size_t)hq * r * D;
   for (int c = tid; c < D; c += NT) s_q[c] = __bfloat162float(qp[c]);
   if (p.mlp_q.w_s != nullptr) {
+    const float* a = p.mlp_vec + (size_t)row * (3 * p.mlp_q.d_emb + r) + 3 * p.mlp_q.d_emb;
+    if (tid < r) s_a[tid] = __ldcg(a + tid);
     __syncthreads();
-    mlp_phi_q_log<NT>(p, hq, s_q, mlp_scratch, s_a);
     float m = -INFINITY;
     for (int j = lane; j < r; j += 32) m = fmaxf(m, s_a[j]);
     m = warp_max(m);

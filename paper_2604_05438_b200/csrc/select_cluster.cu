@@ -99,7 +99,7 @@ select_kernel(const Problem p, const int n_rows, const int csize) {
     pdl_wait();                                            // the workspace is free once the predecessors are done
     const int task = ((int)blockIdx.y - n_rows) * csize + (int)blockIdx.x;
     if (task < n_rows) {
-      phi_q_stage1<kSelThreads>(p, task, reinterpret_cast<float*>(keys_s));   // (a feature CTA holds no keys)
+      phi_q_stage1<kSelThreads>(p, task);
       __threadfence_block();
       __syncthreads();
       phi_q_stage2<kSelThreads>(p, task);
