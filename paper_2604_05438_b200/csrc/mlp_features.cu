@@ -2,19 +2,19 @@
 //   g0 = W_s x + b_s;  Delta = W_2 GeLU(W_1 g0 + b_1) + b_2;  g1 = g0 + alpha Delta;  phi(x) = exp(W_o g1 + b_o).
 // Key side: phi_k of every cache row is four dense layers over all tokens, i.e. four GEMMs per KV head
 // ([tokens x K] . [N x K]^T); they run on the tensor cores (tcgen05.mma, accumulators in tensor memory,
-// both operands staged by TMA into a 3-stage ring), each followed by its layer's epilogue (bias,
+// both operands staged by TMA into a 2-stage ring, three CTAs per SM), each followed by its layer's epilogue (bias,
 // GeLU, the gated residual, the exponential).  Activations between the layers are bf16 in the caller's
 // workspace; accumulation, biases and the exponent are fp32.  The rows of phi_k go to the caller's
 // feature cache, from which the summaries are built (build_summaries.cu, cached variant) and the
 // decode step takes the retrieved tokens' rows (cached_features.cu).
-// Query side: one vector per head and decode step: see mlp_phi_q in feature_jobs.cuh.
+// Query side: one vector per head and decode step: mlp_query.cu.
 #include "common.cuh"
 #include "sm100.cuh"
 
 namespace tkphi {
 
-constexpr int kGemmThreads = 192;      // warp 0: TMA producer, warp 1: MMA issuer, warps 2..5: epilogue
-constexpr int kGemmStages = 3;
+constexpr int kGemmThreads = 320;      // warp 0: TMA producer, warp 1: MMA issuer, warps 2..9: epilogue (two per lane quadrant)
+constexpr int kGemmStages = 2;
 constexpr int kGemmBM = 128;           // rows (tokens) per CTA = MMA M = tensor-memory lanes
 constexpr int kGemmBK = 64;            // reduction elements per stage: one 128-byte swizzled row
 
@@ -88,15 +88,16 @@ mlp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (ok) tc_commit(done);
     }
   } else {
-    // ---- epilogue: thread = output row (tensor-memory lane 32 (warp % 4) + lane)
-    const int quad = warp & 3, row = quad * 32 + lane, m = m0 + row;
+    // ---- epilogue: thread = output row (tensor-memory lane 32 (warp % 4) + lane) x one half of the columns
+    const int quad = warp & 3, half = (warp - 2) >> 2, row = quad * 32 + lane, m = m0 + row;
     const bool ok = __all_sync(0xffffffffu, mbar_wait(done, 0, s_abort));
     if (ok) {
       tc_fence_after_sync();
       const float al = g.epi == kEpiResidual ? g.alpha[h] : 0.f;
       const size_t o = (size_t)h * g.out_head_stride + (size_t)m * g.N + n0;
 #pragma unroll
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int cc = 0; cc < BN / 64; ++cc) {
+        const int c = half * (BN / 64) + cc;
         float v[32];
         tmem_ld_x32(tmem_addr(tmem_base, quad * 32, c * 32), v);
         tc_wait_ld();
