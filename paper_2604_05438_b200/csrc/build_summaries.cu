@@ -12,7 +12,7 @@
 //            the key tile as TMA lands it.  The fp32 result sits in tensor memory with one
 //            feature per lane and one token per column.
 //   features Phi^T[j][t] = exp2(A^T + b_j - gamma |k_t|^2) (everything pre-scaled by
-//            log2 e).  Eight warps read the accumulator into registers, add u_j += Phi
+//            log2 e).  The feature warps read the accumulator into registers, add u_j += Phi
 //            (fp32), split Phi into bf16 hi + lo (error ~2^-17) and store both over the
 //            accumulator columns they have read, as A operands (two tokens per column).
 //            There are two such accumulator / operand buffers, used by alternate tiles.
@@ -30,8 +30,10 @@
 // the two GEMMs of a tile was idle time of the tensor pipe).
 // Key and value tiles share one ring of shared-memory slots, filled in the order in which the
 // tensor pipe consumes them.  GEMM 1 of tile i+1 runs into the other buffer while the feature
-// warps work on tile i, so the tensor pipe works while the feature warps are busy.  Each CTA owns a contiguous range of tiles of one
-// (sequence, KV head) unit and writes one partial; a second small kernel adds the
+// warps work on tile i, so the tensor pipe works while the feature warps are busy.  Each CTA
+// owns a contiguous range of tiles of one (sequence, KV head) unit (at most 256 tiles, which also
+// bounds the rounding bias of a tensor-memory accumulation chain) and writes one partial; a second
+// small kernel, launched as a programmatic dependent, adds the
 // partials in chunk order.  Every device-side wait is bounded and reports through the
 // status word.
 #include "common.cuh"
@@ -387,7 +389,7 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
       const bool valid = (t0 + it) * kBT + t < n_mid;
       snorm[buf * 128 + t] = valid ? -g2 * kn : -INFINITY;   // exp2(-inf) = 0 removes rows outside the mid-region
       __syncwarp();
-      if (lane == 0) mbar_arrive(&n_ready[buf]);             // the MMA issuer releases the key slot after this
+      if (lane == 0) mbar_arrive(&n_ready[buf]);             // the GEMM-1 issuer releases the key slot after this
     }
   }
 
