@@ -78,6 +78,10 @@ def test_invalid_arguments_are_rejected_before_any_launch(lib):
     assert _decode(lib, dd, [1]) == -1
     dd, _c = _desc([0, 100], n_sink=0, n_tail=0)
     assert _decode(lib, dd, [0]) == -1 and b"empty exact support" in lib.tkphi_last_error()
+    dd, _c = _desc([0, 2097152 + 4 + 8 + 1])
+    assert _decode(lib, dd, [10]) == -2 and b"2097152" in lib.tkphi_last_error()          # one mid key too many
+    dd, _c = _desc([0, 2097152 + 4 + 8])
+    assert _decode(lib, dd, [10], ws=0) == -3
     # per-sequence tail counts: both pointers or neither, no negative entry; they replace n_tail in every bound
     tails = np.array([8, 90], np.int32)
     dd, _c = _desc([0, 100, 300])

@@ -8,6 +8,8 @@ vanishing share of the mass, and with the visible-residual map (shared random fe
 oracle-calibrated bias shift) under which the residual branch carries an O(1) share, so
 that the subtraction, the residual estimate and the merge are seen by the comparison.
 """
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
@@ -35,9 +37,9 @@ def _phi_for(cfg, inp, seed, kind, frac, samples, dev):
 
 
 def _run_full(cfg_name, frac, samples, seed=0, kind="baseline"):
-    """samples: list of (sequence, query head)."""
+    """samples: list of (sequence, query head); cfg_name: a key of CONFIGS or a WorkloadConfig."""
     import paper_2604_05438_b200 as T
-    cfg = CONFIGS[cfg_name]
+    cfg = CONFIGS[cfg_name] if isinstance(cfg_name, str) else cfg_name
     dev = torch.device("cuda:0")
     inp = make_layer_inputs(cfg, seed, device=dev, n_steps=1)
     phi = _phi_for(cfg, inp, seed, kind, frac, samples, dev)
@@ -137,3 +139,9 @@ def test_c4_ragged_32_sequences_sampled(kind):
 def test_c5_four_sequences_of_one_million_tokens_sampled(kind):
     # eight rows over three (sequence, KV head) pairs
     _run_full("c5_3b_1m", 0.01, [(0, 6), (0, 7), (0, 8), (3, 18), (3, 19), (3, 20), (1, 0), (1, 1)], kind=kind)
+
+
+def test_longest_supported_sequence_2097152_mid_keys():
+    # the documented limit of the selection kernel (16 rounds per CTA of an 8-CTA cluster); two KV heads
+    cfg = dataclasses.replace(CONFIGS["c1_1b_4k"], n_q_heads=4, n_kv_heads=2, seq_len=2097152 + 4 + 64, needles_per_head=8)
+    _run_full(cfg, 0.001, [(0, 1), (0, 2)], seed=3, kind="baseline")
