@@ -27,17 +27,31 @@ __global__ void __launch_bounds__(kZThreads) cached_z_kernel(const Problem p) {
   const int* idx = p.idx + (size_t)row * p.topk_max;
   float* z = p.zbuf + (size_t)row * p.topk_max;
   const int per_block = (kZThreads / 32) * RPW;
-  for (int i0 = blockIdx.x * per_block + warp * RPW; i0 < K; i0 += gridDim.x * per_block) {
-    const int i = i0 + lane / LPR;
-    float acc = 0.f;
-    if (i < K) {
-      const int ti = __ldcg(idx + i);
-      const float4 f = __ldcs(reinterpret_cast<const float4*>(fbase + (size_t)ti * R) + lane % LPR);
-      acc = fmaf(w.x, f.x, fmaf(w.y, f.y, fmaf(w.z, f.z, w.w * f.w)));
+  const int stride = gridDim.x * per_block;
+  constexpr int U = 4;                           // tokens in flight per warp slot: the index and row loads are latency-bound
+  for (int i0 = blockIdx.x * per_block + warp * RPW; i0 < K; i0 += U * stride) {
+    int ti[U];
+    float acc[U];
+#pragma unroll
+    for (int n = 0; n < U; ++n) {
+      const int i = i0 + n * stride + lane / LPR;
+      ti[n] = i < K ? __ldcg(idx + i) : -1;
     }
 #pragma unroll
-    for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (i < K && lane % LPR == 0) z[i] = acc;
+    for (int n = 0; n < U; ++n) {
+      acc[n] = 0.f;
+      if (ti[n] >= 0) {
+        const float4 f = __ldcs(reinterpret_cast<const float4*>(fbase + (size_t)ti[n] * R) + lane % LPR);
+        acc[n] = fmaf(w.x, f.x, fmaf(w.y, f.y, fmaf(w.z, f.z, w.w * f.w)));
+      }
+    }
+#pragma unroll
+    for (int n = 0; n < U; ++n) {
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) acc[n] += __shfl_xor_sync(0xffffffffu, acc[n], o);
+      const int i = i0 + n * stride + lane / LPR;
+      if (i < K && lane % LPR == 0) z[i] = acc[n];
+    }
   }
 }
 
