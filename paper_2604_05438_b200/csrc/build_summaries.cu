@@ -3,19 +3,18 @@
 //   phi_k(k) = exp(W_k k + b_k - gamma_k |k|^2).
 //
 // Both contractions of the build are dense, so both run on the tensor cores
-// (tcgen05.mma, accumulators in tensor memory).  Everything but the key and value tiles lives
-// in tensor memory, so that shared memory -- whose bandwidth the MMA operand reads, the TMA
-// writes and the norm reads share -- carries each tile only as often as it must, and all of
-// it is left to the key/value stream.  Per tile of 128 mid-region tokens:
+// (tcgen05.mma, accumulators in tensor memory).  The features never leave tensor memory: they
+// are written over the accumulator they were computed from and read from there as the A
+// operand of the second GEMM.  Per tile of 128 mid-region tokens:
 //   GEMM 1   A^T[j][t] = sum_c W_k[j][c] k_t[c]      A operand: W_k (split into bf16
-//            hi + lo, rows = features, zero padded to 128) from tensor memory, B operand:
+//            hi + lo, rows = features, zero padded to 128) in shared memory, B operand:
 //            the key tile as TMA lands it.  The fp32 result sits in tensor memory with one
 //            feature per lane and one token per column.
 //   features Phi^T[j][t] = exp2(A^T + b_j - gamma |k_t|^2) (everything pre-scaled by
 //            log2 e).  The feature warps read the accumulator into registers, add u_j += Phi
 //            (fp32), split Phi into bf16 hi + lo (error ~2^-17) and store both over the
 //            accumulator columns they have read, as A operands (two tokens per column).
-//            There are two such accumulator / operand buffers, used by alternate tiles.
+//            There are three such accumulator / operand buffers, used by the tiles in turn.
 //   GEMM 2   S^T[j][c] += sum_t Phi^T[j][t] v_t[c]   A operand: Phi^T hi, then lo, from
 //            tensor memory; B operand: the value tile as TMA lands it (MN-major: dims
 //            contiguous, tokens along K).  S^T accumulates in tensor memory over all tiles
@@ -29,8 +28,9 @@
 // issuing thread advances only as fast as its MMAs execute, so with one issuer every barrier wait between
 // the two GEMMs of a tile was idle time of the tensor pipe).
 // Key and value tiles share one ring of shared-memory slots, filled in the order in which the
-// tensor pipe consumes them.  GEMM 1 of tile i+1 runs into the other buffer while the feature
-// warps work on tile i, so the tensor pipe works while the feature warps are busy.  Each CTA
+// tensor pipe consumes them.  GEMM 1 of tiles i+1 and i+2 runs into the other buffers while the
+// feature warps work on tile i and GEMM 2 of tile i waits for them, so the tensor pipe works
+// while the feature warps are busy.  Each CTA
 // owns a contiguous range of tiles of one (sequence, KV head) unit (at most 256 tiles, which also
 // bounds the rounding bias of a tensor-memory accumulation chain) and writes one partial; a second
 // small kernel, launched as a programmatic dependent, adds the
@@ -49,10 +49,10 @@ constexpr int kWarpG2 = kWarpNorm + 4;   // GEMM-2 issuer
 constexpr int kBuildThreads = (kWarpG2 + 1) * 32;
 constexpr int kBT = 128;                 // tokens per tile
 constexpr int kBuildTmemCols = 512;
-constexpr int kColW = 0;                 // W_k as the A operand of GEMM 1: 64 packed columns hi, then 64 lo
-constexpr int kColBuf = 128;             // two buffers of 128 columns: GEMM-1 accumulator, then Phi^T hi / lo as the A operand
+constexpr int kNB = 3;                   // accumulator / operand buffers in tensor memory
+constexpr int kColBuf = 0;               // kNB buffers of 128 columns: GEMM-1 accumulator, then Phi^T hi / lo as the A operand
                                          // of GEMM 2 (per token group of a feature thread: its packed columns hi, then lo)
-constexpr int kColD2 = 384;              // S^T accumulator, head_dim columns
+constexpr int kColD2 = kNB * 128;        // S^T accumulator, head_dim columns
 
 __device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
@@ -68,11 +68,13 @@ struct BuildCfg {
   static constexpr int BOXES = D / 64;
   static constexpr int BOX = kBT * 128;                    // bytes of one 64-dim column block of a tile
   static constexpr int TILE = BOXES * BOX;                 // 32 KB (d = 128) or 16 KB (d = 64)
-  static constexpr int NS = D == 128 ? 7 : 10;             // slots of the key/value ring (2 NS + 10 barriers <= 32)
-  static constexpr size_t ring = 0;
+  static constexpr int NS = D == 128 ? 5 : 10;             // slots of the key/value ring (2 NS + 4 kNB + 2 barriers <= 40)
+  static constexpr size_t whi = 0;                         // W_k hi / lo operand tiles: 128 feature rows x D dims, swizzled
+  static constexpr size_t wlo = whi + TILE;
+  static constexpr size_t ring = wlo + TILE;
   static constexpr size_t small = ring + (size_t)NS * TILE;
-  // small: barriers (<= 32), snorm[2][128], misc; the per-group feature sums reuse the ring at the end
-  static constexpr size_t total = small + 32 * 8 + 4 * (2 * 128 + 16);
+  // small: barriers (<= 40), snorm[kNB][128], misc; the per-group feature sums reuse the ring at the end
+  static constexpr size_t total = small + 40 * 8 + 4 * (kNB * 128 + 16);
 };
 
 // MODE 0: features computed; 1: computed and also stored to the feature cache; 2: read from the
@@ -85,19 +87,21 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   constexpr int NS = C::NS, BOXES = C::BOXES;
   constexpr int LPT = MODE == 2 ? 1 : 2;       // ring loads per tile
   extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* whi = smem + C::whi;
+  unsigned char* wlo = smem + C::wlo;
   unsigned char* ring = smem + C::ring;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::small);
   uint64_t* full = bars;                   // [NS] tile landed
   uint64_t* empty = full + NS;             // [NS] the MMAs that read the slot are complete (and, for a key tile, its norms taken)
-  uint64_t* d1_full = empty + NS;          // [2]  GEMM 1 accumulator complete
-  uint64_t* buf_free = d1_full + 2;        // [2]  GEMM 2 of the tile is complete: its buffer may take the next accumulator
-  uint64_t* p_ready = buf_free + 2;        // [2]  feature operand of the tile stored to tensor memory
-  uint64_t* n_ready = p_ready + 2;         // [2]  key norms of the tile in shared memory
-  uint64_t* d2_full = n_ready + 2;         // [1]  last GEMM 2 complete
-  uint64_t* w_ready = d2_full + 1;         // [1]  W_k operand stored to tensor memory
-  float* snorm = reinterpret_cast<float*>(bars + 32);        // [2][128]  -gamma log2e |k_t|^2, -inf if masked
+  uint64_t* d1_full = empty + NS;          // [kNB]  GEMM 1 accumulator complete
+  uint64_t* buf_free = d1_full + kNB;      // [kNB]  GEMM 2 of the tile is complete: its buffer may take the next accumulator
+  uint64_t* p_ready = buf_free + kNB;      // [kNB]  feature operand of the tile stored to tensor memory
+  uint64_t* n_ready = p_ready + kNB;       // [kNB]  key norms of the tile in shared memory
+  uint64_t* d2_full = n_ready + kNB;       // [1]  last GEMM 2 complete
+  uint64_t* w_ready = d2_full + 1;         // [1]  W_k operand tiles converted
+  float* snorm = reinterpret_cast<float*>(bars + 40);        // [kNB][128]  -gamma log2e |k_t|^2, -inf if masked
   float* ucomb = reinterpret_cast<float*>(ring);             // [kNG][128], written after the last MMA has read the ring
-  int* misc = reinterpret_cast<int*>(snorm + 2 * 128);
+  int* misc = reinterpret_cast<int*>(snorm + kNB * 128);
   volatile int* s_abort = misc;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc + 1);
 
@@ -132,14 +136,14 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   auto seq_v = [&](int i) { return MODE == 2 ? i : (2 * i + 2 < 2 * n_my - 1 ? 2 * i + 2 : 2 * n_my - 1); };
 
   // ---- set-up: barriers and tensor memory first, so that the producer can start the key/value
-  // stream while four warps (one per lane quadrant) store W_k (scaled by log2 e, hi + lo) to tensor memory
+  // stream while the other warps convert the W_k operand tiles (scaled by log2 e, hi + lo)
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < kNB; ++s) {
       mbar_init(&p_ready[s], kFWarps); mbar_init(&n_ready[s], 4); mbar_init(&d1_full[s], 1); mbar_init(&buf_free[s], 1);
     }
     mbar_init(d2_full, 1);
-    mbar_init(w_ready, 4 * (D / 32) <= kFWarps ? 4 * (D / 32) : 4);
+    mbar_init(w_ready, kBuildThreads / 32 - 1);
     mbar_fence_init();
     *s_abort = 0;
   }
@@ -148,34 +152,30 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
-  // one warp per (lane quadrant, block of 32 dims) when there are enough feature warps, else one per quadrant
-  constexpr bool kSplitW = 4 * (D / 32) <= kFWarps;
-  if (MODE != 2 && warp >= 2 && warp < 2 + (kSplitW ? 4 * (D / 32) : 4)) {
-    // thread = feature row j (tensor-memory lane); column c of the operand holds dims 2c, 2c + 1
-    const int j = (warp & 3) * 32 + lane;
-    const float* Wj = p.w_k + ((size_t)kvh * R + (j < R ? j : 0)) * D;
-    const int blk0 = kSplitW ? (warp - 2) >> 2 : 0, blk1 = kSplitW ? blk0 + 1 : D / 32;
-    for (int blk = blk0; blk < blk1; ++blk) {              // 32 dims -> 16 packed columns
-      uint32_t hw[16], lw[16];
+  if (MODE != 2 && warp != 0) {
+    const float* W = p.w_k + (size_t)kvh * R * D;
+    constexpr int CPR = D / 8;
+    for (int i = tid - 32; i < 128 * CPR; i += kBuildThreads - 32) {
+      const int row = i / CPR, c = i % CPR;
+      unsigned hw[4] = {0, 0, 0, 0}, lw[4] = {0, 0, 0, 0};
+      if (row < R) {
+        const float4 w0 = __ldg(reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8));
+        const float4 w1 = __ldg(reinterpret_cast<const float4*>(W + (size_t)row * D + c * 8 + 4));
+        const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
-      for (int f = 0; f < 8; ++f) {
-        float4 w4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j < R) w4 = __ldg(reinterpret_cast<const float4*>(Wj + blk * 32 + f * 4));
-        const float w[4] = {w4.x * kLog2e, w4.y * kLog2e, w4.z * kLog2e, w4.w * kLog2e};
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const __nv_bfloat162 hp = __floats2bfloat162_rn(w[2 * e], w[2 * e + 1]);      // .x (low half) = even dim
-          const __nv_bfloat162 lp =
-              __floats2bfloat162_rn(w[2 * e] - __bfloat162float(hp.x), w[2 * e + 1] - __bfloat162float(hp.y));
-          hw[2 * f + e] = *reinterpret_cast<const uint32_t*>(&hp);
-          lw[2 * f + e] = *reinterpret_cast<const uint32_t*>(&lp);
+        for (int e = 0; e < 4; ++e) {
+          const float a0 = w[2 * e] * kLog2e, a1 = w[2 * e + 1] * kLog2e;
+          const __nv_bfloat162 hp = __floats2bfloat162_rn(a0, a1);
+          const __nv_bfloat162 lp = __floats2bfloat162_rn(a0 - __bfloat162float(hp.x), a1 - __bfloat162float(hp.y));
+          hw[e] = *reinterpret_cast<const uint32_t*>(&hp);
+          lw[e] = *reinterpret_cast<const uint32_t*>(&lp);
         }
       }
-      tmem_st_x16(tmem_addr(tmem_base, (warp & 3) * 32, kColW + blk * 16), hw);
-      tmem_st_x16(tmem_addr(tmem_base, (warp & 3) * 32, kColW + 64 + blk * 16), lw);
+      const uint32_t off = (c >> 3) * C::BOX + swz128(row, c & 7);
+      *reinterpret_cast<uint4*>(whi + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      *reinterpret_cast<uint4*>(wlo + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
     }
-    tc_wait_st();
-    tc_fence_before_sync();
+    fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) mbar_arrive(w_ready);
   }
@@ -218,27 +218,30 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     if (MODE != 2 && lane == 0) {
       constexpr uint32_t idesc1 = umma_idesc_bf16(128, kBT, 0, 0);
       const uint64_t ring_k = umma_smem_desc(smem_u32(ring), 16, 1024);
+      const uint64_t whi_d = umma_smem_desc(smem_u32(whi), 16, 1024);
+      const uint64_t wlo_d = umma_smem_desc(smem_u32(wlo), 16, 1024);
       bool ok = mbar_wait(w_ready, 0, s_abort);
       tc_fence_after_sync();
       for (int it = 0; it < n_my && ok; ++it) {
-        const int buf = it & 1, nk = seq_k(it), ks = nk % NS;
-        // the buffer is free once GEMM 2 of tile it-2 has read its features
+        const int buf = it % kNB, nk = seq_k(it), ks = nk % NS;
+        // the buffer is free once GEMM 2 of tile it - kNB has read its features
         ok = mbar_wait(&full[ks], (uint32_t)(nk / NS) & 1u, s_abort) &&
-             (it < 2 || mbar_wait(&buf_free[buf], (uint32_t)((it - 2) >> 1) & 1u, s_abort));
+             (it < kNB || mbar_wait(&buf_free[buf], (uint32_t)(it / kNB - 1) & 1u, s_abort));
         if (!ok) break;
         tc_fence_after_sync();
         const uint64_t kd = ring_k + (uint64_t)((ks * C::TILE) >> 4);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
+          const uint64_t wd = half == 0 ? whi_d : wlo_d;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint64_t off = (uint64_t)(((k >> 2) * C::BOX + (k & 3) * 32) >> 4);
-            umma_ts(tmem_base + kColBuf + buf * 128, tmem_base + kColW + half * 64 + k * 8, kd + off, idesc1, (half | k) ? 1u : 0u);
+            umma_ss(tmem_base + kColBuf + buf * 128, wd + off, kd + off, idesc1, (half | k) ? 1u : 0u);
           }
         }
         tc_commit(&d1_full[buf]);
         // the slot is released once GEMM 1 is complete and the norm warps have read the tile
-        ok = mbar_wait(&n_ready[buf], (uint32_t)(it >> 1) & 1u, s_abort);
+        ok = mbar_wait(&n_ready[buf], (uint32_t)(it / kNB) & 1u, s_abort);
         if (!ok) break;
         tc_commit(&empty[ks]);
       }
@@ -252,8 +255,8 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
       const uint64_t ring_v = umma_smem_desc(smem_u32(ring), C::BOX, 1024);
       bool ok = true;
       for (int j = 0; j < n_my && ok; ++j) {
-        const int buf = j & 1, nv = seq_v(j), vs = nv % NS;
-        ok = mbar_wait(&p_ready[buf], (uint32_t)(j >> 1) & 1u, s_abort) &&
+        const int buf = j % kNB, nv = seq_v(j), vs = nv % NS;
+        ok = mbar_wait(&p_ready[buf], (uint32_t)(j / kNB) & 1u, s_abort) &&
              mbar_wait(&full[vs], (uint32_t)(nv / NS) & 1u, s_abort);
         if (!ok) break;
         tc_fence_after_sync();
@@ -282,10 +285,10 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     float* cache_j = (MODE != 0 && j < R) ? p.phi_cache + ((size_t)kvh * p.total_tokens + (size_t)row0) * R + j : nullptr;
     bool ok = true;
     for (int it = 0; it < n_my && ok; ++it) {
-      const int buf = it & 1;
-      const uint32_t ph = (uint32_t)(it >> 1) & 1u;
+      const int buf = it % kNB;
+      const uint32_t ph = (uint32_t)(it / kNB) & 1u;
       // mode 2 has no GEMM 1 whose issuer would wait for the buffer
-      ok = (MODE == 2 ? (it < 2 || mbar_wait(&buf_free[buf], (uint32_t)((it - 2) >> 1) & 1u, s_abort))
+      ok = (MODE == 2 ? (it < kNB || mbar_wait(&buf_free[buf], (uint32_t)(it / kNB - 1) & 1u, s_abort))
                       : mbar_wait(&d1_full[buf], ph, s_abort)) &&
            mbar_wait(&n_ready[buf], ph, s_abort);
       ok = __all_sync(0xffffffffu, ok);
@@ -367,10 +370,10 @@ build_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__
     const float g2 = p.gamma_k * kLog2e;
     bool ok = true;
     for (int it = 0; it < n_my && ok; ++it) {
-      const int buf = it & 1, nk = seq_k(it), ks = nk % NS;
-      // snorm[buf] was last read by the feature warps for tile it-2: wait for their p_ready
+      const int buf = it % kNB, nk = seq_k(it), ks = nk % NS;
+      // snorm[buf] was last read by the feature warps for tile it - kNB: wait for their p_ready
       ok = (MODE == 2 || mbar_wait(&full[ks], (uint32_t)(nk / NS) & 1u, s_abort)) &&
-           mbar_wait(&p_ready[buf], ((uint32_t)(it >> 1) & 1u) ^ 1u, s_abort);
+           mbar_wait(&p_ready[buf], ((uint32_t)(it / kNB) & 1u) ^ 1u, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       const unsigned char* tile = ring + ks * C::TILE;
