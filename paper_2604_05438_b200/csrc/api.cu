@@ -448,9 +448,13 @@ tkphi_status decode_common(const tkphi_kv_desc* kv, const tkphi_phi_desc* phi, c
     memset(&gk, 0, sizeof(gk));
     memset(&gv, 0, sizeof(gv));
     long long ratio_v = 0, rows_v = 0;
-    p.gather_mode = make_gather_map(kv, kv->k, sh.total_tokens, &gk, &p.gather_ratio, &p.gather_rows);
-    if (p.gather_mode >= 0 && make_gather_map(kv, kv->v, sh.total_tokens, &gv, &ratio_v, &rows_v) != p.gather_mode)
-      p.gather_mode = -1;
+    // the row-gather maps are needed (and encoded) only where the streaming kernel can be chosen
+    p.gather_mode = -1;
+    if (n_pairs > n_sm_cached() && kv->head_dim == 128) {
+      p.gather_mode = make_gather_map(kv, kv->k, sh.total_tokens, &gk, &p.gather_ratio, &p.gather_rows);
+      if (p.gather_mode >= 0 && make_gather_map(kv, kv->v, sh.total_tokens, &gv, &ratio_v, &rows_v) != p.gather_mode)
+        p.gather_mode = -1;
+    }
     e = launch_exact_residual(p, gk, gv, n_pairs, n_sm_cached(), cs);
   }
   if (e != cudaSuccess) return cuda_fail(e, "exact_residual launch");
