@@ -604,29 +604,29 @@ tkphi_status tkphi_mlp_key_features(const tkphi_kv_desc* kv, const tkphi_mlp_des
   if (e != cudaSuccess) return cuda_fail(e, "weight conversion launch");
   // tensor maps: activations [head][token][k] (the keys through the cache's own strides), weights [head][n][k]
   CUtensorMap a_k, a_g0, a_h, a_g1, m_ws, m_w1, m_w2, m_wo;
-  const int bn_o = R % 128 == 0 ? 128 : 64;
+  const int bn_e = mlp_gemm_bn(E), bn_o = mlp_gemm_bn(R);
   if ((st = make_tensor_map(kv, kv->k, 128, T, &a_k)) != TKPHI_OK) return st;
   if ((st = make_gemm_map(g0, E, T, H, E, T * E, 128, &a_g0)) != TKPHI_OK) return st;
   if ((st = make_gemm_map(hb, E, T, H, E, T * E, 128, &a_h)) != TKPHI_OK) return st;
   if ((st = make_gemm_map(g1, E, T, H, E, T * E, 128, &a_g1)) != TKPHI_OK) return st;
-  if ((st = make_gemm_map(ws_, D, E, H, D, (long long)E * D, 128, &m_ws)) != TKPHI_OK) return st;
-  if ((st = make_gemm_map(w1_, E, E, H, E, (long long)E * E, 128, &m_w1)) != TKPHI_OK) return st;
-  if ((st = make_gemm_map(w2_, E, E, H, E, (long long)E * E, 128, &m_w2)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(ws_, D, E, H, D, (long long)E * D, bn_e, &m_ws)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(w1_, E, E, H, E, (long long)E * E, bn_e, &m_w1)) != TKPHI_OK) return st;
+  if ((st = make_gemm_map(w2_, E, E, H, E, (long long)E * E, bn_e, &m_w2)) != TKPHI_OK) return st;
   if ((st = make_gemm_map(wo_, E, R, H, E, (long long)R * E, bn_o, &m_wo)) != TKPHI_OK) return st;
   GemmArgs g{};
-  g.M = (int)T; g.status = status;
+  g.M = (int)T; g.heads = H; g.status = status;
   // g0 = W_s x + b_s
   g.N = E; g.K = D; g.epi = kEpiBias; g.bias = mlp_k->b_s; g.out = g0; g.out_head_stride = T * E;
-  if ((e = launch_mlp_gemm(a_k, m_ws, g, H, cs)) != cudaSuccess) return cuda_fail(e, "MLP stem launch");
+  if ((e = launch_mlp_gemm(a_k, m_ws, g, cs)) != cudaSuccess) return cuda_fail(e, "MLP stem launch");
   // h = GeLU(W_1 g0 + b_1)
   g.K = E; g.epi = kEpiGelu; g.bias = mlp_k->b_1; g.out = hb;
-  if ((e = launch_mlp_gemm(a_g0, m_w1, g, H, cs)) != cudaSuccess) return cuda_fail(e, "MLP layer 1 launch");
+  if ((e = launch_mlp_gemm(a_g0, m_w1, g, cs)) != cudaSuccess) return cuda_fail(e, "MLP layer 1 launch");
   // g1 = g0 + alpha (W_2 h + b_2)
   g.epi = kEpiResidual; g.bias = mlp_k->b_2; g.alpha = mlp_k->alpha; g.resid = g0; g.out = g1;
-  if ((e = launch_mlp_gemm(a_h, m_w2, g, H, cs)) != cudaSuccess) return cuda_fail(e, "MLP layer 2 launch");
+  if ((e = launch_mlp_gemm(a_h, m_w2, g, cs)) != cudaSuccess) return cuda_fail(e, "MLP layer 2 launch");
   // phi = exp(W_o g1 + b_o)
   g.N = R; g.epi = kEpiExp; g.bias = mlp_k->b_o; g.out = phi_k_cache; g.out_head_stride = T * R;
-  if ((e = launch_mlp_gemm(a_g1, m_wo, g, H, cs)) != cudaSuccess) return cuda_fail(e, "MLP output layer launch");
+  if ((e = launch_mlp_gemm(a_g1, m_wo, g, cs)) != cudaSuccess) return cuda_fail(e, "MLP output layer launch");
   return TKPHI_OK;
 }
 

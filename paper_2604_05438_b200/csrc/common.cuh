@@ -215,7 +215,7 @@ cudaError_t launch_mlp_query(const Problem& p, cudaStream_t stream);
 // out[h][m][n] = epilogue(sum_k A[h][m][k] W[h][n][k] + bias[h][n]).
 enum { kEpiBias = 0, kEpiGelu = 1, kEpiResidual = 2, kEpiExp = 3 };
 struct GemmArgs {
-  int M, N, K;                         // rows, output columns, reduction length (K a multiple of 64)
+  int M, N, K, heads;                  // rows, output columns, reduction length (K a multiple of 64), matrix sets
   int epi;
   const float* bias;                   // [heads][N]
   const float* alpha;                  // [heads] (kEpiResidual)
@@ -224,7 +224,9 @@ struct GemmArgs {
   long long out_head_stride;           // elements between heads of out (and of resid)
   int* status;
 };
-cudaError_t launch_mlp_gemm(const CUtensorMap& map_a, const CUtensorMap& map_w, const GemmArgs& g, int heads, cudaStream_t stream);
+// Output columns per tile of the MLP GEMM kernel (also the row count of the weight tensor map's box).
+inline int mlp_gemm_bn(int N) { return N % 256 == 0 ? 256 : N % 128 == 0 ? 128 : N == 64 ? 64 : 0; }
+cudaError_t launch_mlp_gemm(const CUtensorMap& map_a, const CUtensorMap& map_w, const GemmArgs& g, cudaStream_t stream);
 cudaError_t launch_f32_to_bf16(const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t stream);
 cudaError_t launch_build(const BuildProblem& p, const CUtensorMap& tmap_k, const CUtensorMap& tmap_v, cudaStream_t stream);
 
