@@ -14,7 +14,7 @@
 
 namespace tkphi {
 
-constexpr int kGemmThreads = 320;      // warp 0: TMA producer, warp 1: MMA issuer, warps 2..9: epilogue (two per lane quadrant)
+constexpr int kGemmThreads = 576;      // warp 0: TMA producer, warp 1: MMA issuer, warps 2..17: epilogue (four per lane quadrant)
 constexpr int kGemmBM = 128;           // rows (tokens) per tile = MMA M = tensor-memory lanes
 constexpr int kGemmBK = 64;            // reduction elements per stage: one 128-byte swizzled row
 
@@ -109,9 +109,11 @@ mlp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       }
     }
   } else {
-    // ---- epilogue: thread = output row (tensor-memory lane 32 (warp % 4) + lane) x one half of the columns
-    const int quad = warp & 3, half = (warp - 2) >> 2, row = quad * 32 + lane;
-    constexpr int CH = BN >= 64 ? BN / 64 : 1;             // 32-column chunks per half
+    // ---- epilogue: thread = output row (tensor-memory lane 32 (warp % 4) + lane) x every fourth 32-column chunk
+    // (sixteen warps: the GeLU layer's epilogue is a long dependent chain per element and needs the occupancy)
+    const int quad = warp & 3, sub = (warp - 2) >> 2, row = quad * 32 + lane;
+    constexpr int NCH = BN / 32;                           // chunks of the tile
+    const int last_c = sub + ((NCH - 1 - sub) / 4) * 4;    // this warp's last chunk (sub >= NCH: none)
     bool ok = true;
     long long i = 0;
     for (long long t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++i) {
@@ -123,13 +125,15 @@ mlp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const float al = g.epi == kEpiResidual ? __ldg(g.alpha + h) : 0.f;
       const float* bias = g.bias + (size_t)h * g.N + n0;
       const size_t o = (size_t)h * g.out_head_stride + (size_t)m * g.N + n0;
-#pragma unroll
-      for (int cc = 0; cc < CH; ++cc) {
-        const int c = half * CH + cc;
+      if (sub >= NCH) {                                    // narrow tiles: nothing for this warp to read
+        if (lane == 0) mbar_arrive(&acc_free[acc]);
+        continue;
+      }
+      for (int c = sub; c < NCH; c += 4) {
         float v[32];
         tmem_ld_x32(tmem_addr(tmem_base, quad * 32, acc * ACC_COLS + c * 32), v);
         tc_wait_ld();
-        if (cc == CH - 1) {                                // this warp holds its whole share of the tile in registers
+        if (c == last_c) {                                 // this warp has read its whole share of the tile
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(&acc_free[acc]);
