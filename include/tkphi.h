@@ -265,7 +265,8 @@ tkphi_status tkphi_mlp_key_features(const tkphi_kv_desc* kv, const tkphi_mlp_des
  * Prefill summary build (Sec. 4.1, Eq. natural_cache) from stored key features: S[b][h] = sum_{i in M_b}
  * v_i phi_k(k_i)^T, u[b][h] = sum phi_k(k_i) with phi_k(k_i) read from row cu_seqlens[b] + i of
  * phi_k_cache (as tkphi_mlp_key_features, or tkphi_build_summaries with a cache, wrote it).  kv->k is
- * validated like every descriptor field (a valid device pointer) but its rows are not read.  Outputs, workspace (TKPHI_WS_BUILD) and errors as for tkphi_build_summaries.
+ * validated like every descriptor field (a valid device pointer) but its rows are not read.
+ * Outputs, workspace (TKPHI_WS_BUILD) and errors as for tkphi_build_summaries.
  */
 tkphi_status tkphi_build_summaries_cached(const tkphi_kv_desc* kv, const float* phi_k_cache, float* S, float* u,
                                           void* workspace, size_t workspace_bytes, void* cuda_stream);

@@ -57,7 +57,7 @@ def _calibrate_bo_shift(cfg, inp, pk, pq, frac, kv_heads, n_probe=2):
     return shift
 
 
-def _check_mlp(cfg, seed, seq_lens, frac, heads, d_emb=512, on_device=False):
+def _check_mlp(cfg, seed, seq_lens, frac, heads, d_emb=512, on_device=False, token_major=False):
     """heads: the query heads compared; the oracle runs on their KV heads only."""
     import paper_2604_05438_b200 as T
     dev = torch.device("cuda:0")
@@ -67,7 +67,12 @@ def _check_mlp(cfg, seed, seq_lens, frac, heads, d_emb=512, on_device=False):
     pq = make_mlp_phi_params(cfg, seed, "q", d_emb)
     pk = make_mlp_phi_params(cfg, seed, "k", d_emb)
     pk = make_mlp_phi_params(cfg, seed, "k", d_emb, bo_shift=_calibrate_bo_shift(cfg, inp, pk, pq, frac, kv_heads))
-    kv = T.KVCache(inp.k.to(dev), inp.v.to(dev), inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, inp.n_sink, inp.n_tail)
+    if token_major:   # [row][head][dim] storage, viewed as [head][row][dim]
+        kd = inp.k.permute(1, 0, 2).contiguous().to(dev).permute(1, 0, 2)
+        vd = inp.v.permute(1, 0, 2).contiguous().to(dev).permute(1, 0, 2)
+    else:
+        kd, vd = inp.k.to(dev), inp.v.to(dev)
+    kv = T.KVCache(kd, vd, inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, inp.n_sink, inp.n_tail)
     Hq, Hkv, d, r, B = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_feat, inp.batch
     T_total = int(inp.cu_seqlens[-1])
 
@@ -176,3 +181,9 @@ def test_mlp_phi_one_full_size_128k_layer_sampled_heads():
     # one layer of the 128K workload in its own geometry and anchors; the oracle runs on two KV heads
     cfg = CONFIGS["c3_3b_128k"]
     _check_mlp(cfg, 0, None, 0.01, heads=[3, 4, 5, 21], on_device=True)
+
+
+def test_mlp_phi_hidden_width_384_token_major_cache():
+    # 128-wide GEMM tiles (384 is not a multiple of 256), keys read through a token-major cache layout
+    cfg = dataclasses.replace(CONFIGS["c3_3b_128k"], n_tail=32, n_q_heads=6, n_kv_heads=2)
+    _check_mlp(cfg, 6, [900, 517], 0.03, heads=range(cfg.n_q_heads), d_emb=384, token_major=True)
