@@ -212,6 +212,23 @@ def run_ours(args, rank, world, device):
                 T.decode_step(layers[l][1], phis[l], qs[l], topk, topk_dev, tmax, Ss[l], us[l], None, y_dev[l],
                               None, 0, ws)
 
+    if args.graph:      # the step's launches captured once into a CUDA graph; every step copies its queries in and replays
+        q_graph = torch.empty_like(q_dev[0])
+        step_eager = step
+        step_eager(q_graph.copy_(q_dev[0]))
+        torch.cuda.synchronize()
+        cap = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        prev = torch.cuda.current_stream()
+        with torch.cuda.stream(cap):
+            with torch.cuda.graph(graph, stream=cap):
+                step_eager(q_graph)
+        torch.cuda.set_stream(prev)
+
+        def step(qs):
+            q_graph.copy_(qs, non_blocking=True)
+            graph.replay()
+
     def barrier():
         torch.cuda.synchronize()
         if world > 1:
@@ -237,7 +254,8 @@ def run_ours(args, rank, world, device):
     # ---- per-kernel durations (second pass with the library's event hooks), for the roofline
     kt = None
     if hasattr(T, "kernel_timing"):
-        kt = T.kernel_timing(lambda: [step(q_dev[s % n_q_sets]) for s in range(min(args.steps, 8))])
+        timed_step = step_eager if args.graph else step      # the event hooks fire at launch time, not on a replay
+        kt = T.kernel_timing(lambda: [timed_step(q_dev[s % n_q_sets]) for s in range(min(args.steps, 8))])
 
     # ---- the Top-K baseline path (tkphi_topk_decode: same scoring, selection and exact branch, no residual), timed beside
     def step_topk(qs):
@@ -286,7 +304,7 @@ def run_ours(args, rank, world, device):
         "dtype": "bf16 K/V, f32 accumulate", "data": "synthetic",
         "config": {"workload": workload_string(cfg, n_layers, N, args.budget, tmax, seq_lens),
                    "l2": "inputs (K/V of all layers) exceed L2 by >100x; no flush needed",
-                   "replicas": world, "seed": seed, "phi_k_cache": bool(args.phi_cache or args.mlp_phi),
+                   "replicas": world, "seed": seed, "phi_k_cache": bool(args.phi_cache or args.mlp_phi), "cuda_graph": bool(args.graph),
                    "phi": "one-block ReZero MLP, d_emb 512" if args.mlp_phi else "exp(Wx + b - |x|^2/2)"},
         "step_us": {"median": statistics.median(per_step) * 1e3, "min": min(per_step) * 1e3,
                     "max": max(per_step) * 1e3},
@@ -439,6 +457,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--seq-len", type=int, default=0, help="override the context length (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="launch every layer call eagerly instead of replaying the step's launches from a CUDA graph "
+                         "(captured once from the same library calls; the default)")
     ap.add_argument("--mlp-phi", action="store_true",
                     help="feature maps = the one-block ReZero MLP: key features by tkphi_mlp_key_features into a cache, "
                          "summaries built from the cache, decode steps through tkphi_decode_step_mlp")

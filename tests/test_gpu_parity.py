@@ -388,3 +388,43 @@ def test_results_are_run_to_run_identical():
     a = PU.gpu_decode(gl, inp.q[0], inp.topk(0.02), S, u)
     b = PU.gpu_decode(gl, inp.q[0], inp.topk(0.02), S, u)
     assert np.array_equal(a["y"], b["y"]) and np.array_equal(a["idx"], b["idx"])
+
+
+def test_decode_step_is_capturable_in_a_cuda_graph():
+    """The library allocates nothing and synchronises nothing, so a decode step (three launches chained as
+    programmatic dependents) can be captured once and replayed; the replay gives the eager result bit for bit."""
+    import paper_2604_05438_b200 as T
+    cfg = CONFIGS["c1_1b_4k"]
+    inp = make_layer_inputs(cfg, 21, seq_lens=[3000, 1200], n_steps=2)
+    gl = PU.to_gpu(cfg, inp, make_phi_params(cfg, 21))
+    S, u = PU.gpu_build(gl)
+    dev = gl.dev
+    topk = inp.topk(0.02)
+    tmax = int(topk.max())
+    B, Hq, d = gl.kv.batch, cfg.n_q_heads, cfg.head_dim
+    ws = torch.empty(T.workspace_bytes(gl.kv, topk, tmax, T.WS_DECODE_STEP), dtype=torch.uint8, device=dev)
+    td = torch.from_numpy(topk).to(dev)
+    q = inp.q[0].to(dev).contiguous()
+    y = torch.zeros(B, Hq, d, device=dev)
+    idx = torch.zeros(B, Hq, tmax, dtype=torch.int32, device=dev)
+    T.decode_step(gl.kv, gl.maps, q, topk, td, tmax, S, u, idx, y, None, 0, ws)        # eager (also warms up)
+    torch.cuda.synchronize()
+    y_eager, idx_eager = y.clone(), idx.clone()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            T.decode_step(gl.kv, gl.maps, q, topk, td, tmax, S, u, idx, y, None, 0, ws, stream=stream)
+    y.zero_()
+    idx.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 0
+    assert torch.equal(y, y_eager) and torch.equal(idx, idx_eager)
+    q.copy_(inp.q[1].to(dev))                                                           # new query, same graph
+    graph.replay()
+    torch.cuda.synchronize()
+    y_replay = y.clone()
+    T.decode_step(gl.kv, gl.maps, q, topk, td, tmax, S, u, idx, y, None, 0, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y_replay)
