@@ -184,9 +184,24 @@ def run_ours(args, rank, world, device):
         build_one = lambda l: T.build_summaries(layers[l][1], phis[l], Ss[l], us[l], wsb)
     build_one(0)                                                     # warm-up
     torch.cuda.synchronize()
+
+    def build_all():
+        for l in range(n_layers):
+            build_one(l)
+
+    if args.graph:      # as for the decode steps: the calls captured once, the graph replayed
+        cap_b = torch.cuda.Stream()
+        graph_b = torch.cuda.CUDAGraph()
+        prev_b = torch.cuda.current_stream()
+        with torch.cuda.stream(cap_b):
+            with torch.cuda.graph(graph_b, stream=cap_b):
+                build_all()
+        torch.cuda.set_stream(prev_b)
+        build_all = graph_b.replay
+        build_all()                                                  # warm-up of the replay
+        torch.cuda.synchronize()
     e0.record()
-    for l in range(n_layers):
-        build_one(l)
+    build_all()
     e1.record()
     torch.cuda.synchronize()
     build_ms = e0.elapsed_time(e1)
