@@ -428,3 +428,54 @@ def test_decode_step_is_capturable_in_a_cuda_graph():
     T.decode_step(gl.kv, gl.maps, q, topk, td, tmax, S, u, idx, y, None, 0, ws)
     torch.cuda.synchronize()
     assert torch.equal(y, y_replay)
+
+
+def test_per_sequence_tails_in_the_streaming_exact_kernel():
+    """Per-sequence tail-anchor counts on a call large enough for the persistent exact/residual kernel
+    (head_dim 128, more slice pairs than SMs): every item of that kernel takes its sequence's own tail."""
+    import paper_2604_05438_b200 as T
+    cfg = _cfg("c3_3b_128k", batch=8, needle_every=256)
+    dev = torch.device("cuda:0")
+    lens = [900, 300, 133, 1500, 700, 2049, 132, 1100]
+    tails = np.array([128, 7, 0, 300, 64, 512, 200, 1], np.int32)
+    inp = make_layer_inputs(cfg, 23, seq_lens=lens, n_steps=1)
+    phi = make_phi_params(cfg, 23, kind="visible", bk_shift=torch.full((cfg.n_kv_heads,), 3.0))
+    kv = T.KVCache(inp.k.to(dev), inp.v.to(dev), inp.cu_seqlens, cfg.n_q_heads, cfg.n_feat, cfg.n_sink, 5, n_tail_seq=tails)
+    pd = phi.to(dev)
+    maps = T.PhiMaps(pd.w_q, pd.b_q, pd.w_k, pd.b_k, pd.gamma_q, pd.gamma_k)
+    B, Hq, Hkv, d, r = 8, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_feat
+    S = torch.full((B, Hkv, d, r), float("nan"), device=dev)
+    u = torch.full((B, Hkv, r), float("nan"), device=dev)
+    wsb = torch.empty(T.workspace_bytes(kv, None, 0, T.WS_BUILD), dtype=torch.uint8, device=dev)
+    T.build_summaries(kv, maps, S, u, wsb)
+    n_mid = np.maximum(0, np.array(lens) - cfg.n_sink - tails)
+    topk = np.floor(0.2 * n_mid).astype(np.int32)
+    tmax = int(topk.max())
+    assert tmax > 256 and int(topk.min()) == 0
+    ws = torch.empty(T.workspace_bytes(kv, topk, tmax, T.WS_DECODE_STEP), dtype=torch.uint8, device=dev)
+    idx = torch.full((B, Hq, tmax), -7, dtype=torch.int32, device=dev)
+    y = torch.full((B, Hq, d), float("nan"), device=dev)
+    dbg = torch.full((B, Hq, 4 + d), float("nan"), device=dev)
+    T.decode_step(kv, maps, inp.q[0].to(dev).contiguous(), topk, torch.from_numpy(topk).to(dev), tmax, S, u, idx, y,
+                  dbg, 0, ws)
+    torch.cuda.synchronize()
+    assert T.device_status(ws) == 0 and T.device_status(wsb) == 0
+    Sh, uh, yh, ih, dh = S.cpu().double().numpy(), u.cpu().double().numpy(), y.cpu().numpy(), idx.cpu().numpy(), dbg.cpu().numpy()
+    for b in range(B):
+        nt = int(tails[b])
+        for hq in range(0, Hq, 5):
+            kvh = hq // cfg.group
+            K, V = PU.seq_arrays(inp, b, kvh)
+            if hq == 0 and n_mid[b] > 0:
+                S0, u0 = O.build_summaries(K, V, phi.w_k[kvh].double().numpy(), phi.b_k[kvh].double().numpy(),
+                                           phi.gamma_k, cfg.n_sink, nt)
+                assert PU.note("S_rel_err", PU.max_rel(Sh[b, kvh], S0)) <= PU.SU_TOL, b
+            q64 = inp.q[0, b, hq].double().numpy()
+            kk = int(topk[b])
+            ret = PU.check_selection(q64, K, cfg.n_sink, nt, kk, ih[b, hq])
+            pa = _phi_arrays(phi, hq, kvh)
+            res = O.topkphi_attention(q64, K, V, cfg.n_sink, nt, kk, *pa, S=Sh[b, kvh], u=uh[b, kvh], retrieved=ret)
+            nosub = O.topkphi_attention(q64, K, V, cfg.n_sink, nt, kk, *pa, S=Sh[b, kvh], u=uh[b, kvh], retrieved=ret,
+                                        subtract=False)
+            assert PU.note("y_rel_err", PU.max_rel(yh[b, hq], res.y)) <= PU.Y_TOL, (b, hq)
+            PU.check_residual(dh[b, hq], res, nosub, (b, hq))
